@@ -1,0 +1,584 @@
+// Host side of the BiTA step library: argument checks, block plans, workspace carving and the
+// launch sequence of one pass.  Every step of the pass runs in the kernels included below.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "attention_simple.cuh"
+#include "common.cuh"
+#include "gemm_simple.cuh"
+#include "step_kernels.cuh"
+
+using namespace bita;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define CU_TRY(expr)                                   \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) {                          \
+      g_last_cuda_error = (int)e__;                    \
+      return BITA_ERR_CUDA;                            \
+    }                                                  \
+  } while (0)
+
+constexpr int PREFILL_CHUNK = 128;
+constexpr size_t ALIGN = 256;
+
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+
+// Host description of a packed block; `upload_plan` writes it into a device region and fills `dev`.
+struct HostPlan {
+  int M = 0, W = 0, N = 0, G = 0, n_mask = 0, k_max = 1, n_query = 0, max_depth = 0;
+  std::vector<int32_t> row_kind, row_idx, rel_pos, parent, rank, depth, group_of;
+  std::vector<uint8_t> sees_prompt;
+  std::vector<uint32_t> vis;
+  DevPlan dev{};
+};
+
+constexpr size_t PLAN_REGION_BYTES =
+    sizeof(int32_t) * (3 * BITA_MAX_ROWS + BITA_MAX_ROWS * (BITA_MAX_ROWS / 32) + 3 * BITA_MAX_NODES +
+                       (BITA_MAX_NODES + 1)) + BITA_MAX_ROWS + 1024;
+
+// Step block (Sec. 3.2, Appendix B): root, tree nodes, G groups of n mask tokens.
+int build_step_plan(const bita_tree_template* t, int n_mask, HostPlan* p) {
+  if (!t || t->N < 0 || t->N > BITA_MAX_NODES || t->G < 0) return BITA_ERR_BAD_TEMPLATE;
+  if (t->N > 0 && (!t->parent || !t->rank)) return BITA_ERR_BAD_TEMPLATE;
+  if (t->G > 0 && !t->attach) return BITA_ERR_BAD_TEMPLATE;
+  if (n_mask < 0 || n_mask > BITA_MAX_MASK) return BITA_ERR_INVALID_ARG;
+  const int N = t->N, G = t->G;
+  const long rows = 1L + N + (long)G * n_mask;
+  if (rows > BITA_MAX_ROWS) return BITA_ERR_BAD_TEMPLATE;
+  p->M = (int)rows;
+  p->W = (p->M + 31) / 32;
+  p->N = N;
+  p->G = G;
+  p->n_mask = n_mask;
+  p->n_query = 0;
+  p->parent.assign(t->parent, t->parent + N);
+  p->rank.assign(t->rank, t->rank + N);
+  p->depth.assign(N, 0);
+  p->k_max = 1;
+  p->max_depth = 0;
+  for (int i = 0; i < N; ++i) {
+    if (p->parent[i] < -1 || p->parent[i] >= i) return BITA_ERR_BAD_TEMPLATE;
+    if (p->rank[i] < 0 || p->rank[i] >= BITA_MAX_TOPK) return BITA_ERR_BAD_TEMPLATE;
+    p->depth[i] = p->parent[i] < 0 ? 1 : p->depth[p->parent[i]] + 1;
+    if (p->depth[i] > BITA_MAX_DEPTH) return BITA_ERR_BAD_TEMPLATE;
+    if (p->depth[i] > p->max_depth) p->max_depth = p->depth[i];
+    if (p->rank[i] + 1 > p->k_max) p->k_max = p->rank[i] + 1;
+  }
+  p->group_of.assign(N + 1, -1);
+  for (int g = 0; g < G; ++g) {
+    const int a = t->attach[g];
+    if (a < -1 || a >= N || p->group_of[a + 1] >= 0) return BITA_ERR_BAD_TEMPLATE;
+    p->group_of[a + 1] = g;
+  }
+  const int M = p->M, W = p->W;
+  p->row_kind.assign(M, ROW_MASK);
+  p->row_idx.assign(M, 0);
+  p->rel_pos.assign(M, 0);
+  p->sees_prompt.assign(M, 0);
+  p->vis.assign((size_t)M * W, 0u);
+  auto set = [&](int r, int c) { p->vis[(size_t)r * W + (c >> 5)] |= 1u << (c & 31); };
+  auto inherit = [&](int r, int from) {
+    for (int w = 0; w < W; ++w) p->vis[(size_t)r * W + w] |= p->vis[(size_t)from * W + w];
+  };
+  p->row_kind[0] = ROW_ROOT;
+  set(0, 0);
+  for (int i = 0; i < N; ++i) {
+    const int r = 1 + i;
+    p->row_kind[r] = ROW_NODE;
+    p->row_idx[r] = i;
+    p->rel_pos[r] = p->depth[i];
+    inherit(r, p->parent[i] + 1);   // the parent's row already holds root..parent
+    set(r, r);
+  }
+  for (int g = 0; g < G; ++g) {
+    const int arow = t->attach[g] + 1;
+    for (int i = 0; i < n_mask; ++i) {
+      const int r = 1 + N + g * n_mask + i;
+      p->row_idx[r] = i;
+      p->rel_pos[r] = p->rel_pos[arow] + i + 1;
+      p->sees_prompt[r] = 1;
+      inherit(r, arow);
+      for (int j = 0; j <= i; ++j) set(r, 1 + N + g * n_mask + j);   // causal inside the group
+    }
+  }
+  return BITA_OK;
+}
+
+// Prefill chunk (Algorithm 1, t = 1): `cnt` query tokens, causal; the last chunk is followed by
+// one group of n_mask mask tokens attached to the final query token.
+void build_prefill_plan(int cnt, int n_mask, bool last, int k_max, HostPlan* p) {
+  const int M = cnt + (last ? n_mask : 0);
+  p->M = M;
+  p->W = (M + 31) / 32;
+  p->N = 0;
+  p->G = last ? 1 : 0;
+  p->n_mask = n_mask;
+  p->k_max = k_max;
+  p->n_query = cnt;
+  p->max_depth = 0;
+  p->parent.clear();
+  p->rank.clear();
+  p->depth.clear();
+  p->group_of.assign(1, -1);
+  p->row_kind.assign(M, ROW_QUERY);
+  p->row_idx.assign(M, 0);
+  p->rel_pos.assign(M, 0);
+  p->sees_prompt.assign(M, 0);
+  p->vis.assign((size_t)M * p->W, 0u);
+  for (int r = 0; r < M; ++r) {
+    p->rel_pos[r] = r;
+    if (r >= cnt) {
+      p->row_kind[r] = ROW_MASK;
+      p->row_idx[r] = r - cnt;
+      p->sees_prompt[r] = 1;
+    } else {
+      p->row_idx[r] = r;
+    }
+    for (int c = 0; c <= r; ++c) p->vis[(size_t)r * p->W + (c >> 5)] |= 1u << (c & 31);
+  }
+}
+
+int upload_plan(HostPlan* p, void* region, cudaStream_t stream) {
+  std::vector<uint8_t> blob(PLAN_REGION_BYTES, 0);
+  size_t off = 0;
+  bool overflow = false;
+  auto put = [&](const void* src, size_t bytes) -> const void* {
+    const size_t at = off;
+    if (at + bytes > PLAN_REGION_BYTES) { overflow = true; return region; }
+    if (bytes) memcpy(blob.data() + at, src, bytes);
+    off = (at + bytes + 15) / 16 * 16;
+    return (const uint8_t*)region + at;
+  };
+  DevPlan& d = p->dev;
+  d.M = p->M; d.W = p->W; d.N = p->N; d.G = p->G; d.n_mask = p->n_mask; d.k_max = p->k_max;
+  d.n_query = p->n_query; d.max_depth = p->max_depth;
+  d.row_kind = (const int32_t*)put(p->row_kind.data(), p->row_kind.size() * 4);
+  d.row_idx = (const int32_t*)put(p->row_idx.data(), p->row_idx.size() * 4);
+  d.rel_pos = (const int32_t*)put(p->rel_pos.data(), p->rel_pos.size() * 4);
+  d.vis = (const uint32_t*)put(p->vis.data(), p->vis.size() * 4);
+  d.parent = (const int32_t*)put(p->parent.data(), p->parent.size() * 4);
+  d.rank = (const int32_t*)put(p->rank.data(), p->rank.size() * 4);
+  d.depth = (const int32_t*)put(p->depth.data(), p->depth.size() * 4);
+  d.group_of = (const int32_t*)put(p->group_of.data(), p->group_of.size() * 4);
+  d.sees_prompt = (const uint8_t*)put(p->sees_prompt.data(), p->sees_prompt.size());
+  if (overflow) return BITA_ERR_BAD_TEMPLATE;
+  CU_TRY(cudaMemcpyAsync(region, blob.data(), off ? off : 16, cudaMemcpyHostToDevice, stream));
+  CU_TRY(cudaStreamSynchronize(stream));
+  return BITA_OK;
+}
+
+int check_dims(const bita_model_dims* m) {
+  if (!m) return BITA_ERR_INVALID_ARG;
+  if (m->L < 1 || m->d < 8 || m->d % 8 || m->H < 1 || m->H_kv < 1 || m->H % m->H_kv) return BITA_ERR_INVALID_ARG;
+  if (m->D != 64 && m->D != 128) return BITA_ERR_INVALID_ARG;
+  if (m->F < 8 || m->F % 8 || m->V < 1 || m->P < 0 || m->P > 64 || m->C_max < 1) return BITA_ERR_INVALID_ARG;
+  if (!(m->rms_eps >= 0.f) || !(m->rope_theta > 0.f)) return BITA_ERR_INVALID_ARG;
+  return BITA_OK;
+}
+
+int attn_splits(int H, int B) {
+  int s = (148 + H * B - 1) / (H * B);
+  if (s < 1) s = 1;
+  if (s > 8) s = 8;
+  return s;
+}
+
+// Device buffers of a context, carved from the caller's workspace.
+struct Buffers {
+  float* x; bf16* xn; float* qkv; bf16* q; bf16* att; float* tmp; float* tmp2; bf16* hf; float* logits;
+  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
+  float2* rope_tab; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
+  int32_t* query_tokens; int32_t* tree_in;
+};
+
+size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> void* {
+    void* p = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return p;
+  };
+  const size_t R = BITA_MAX_ROWS;
+  const size_t nqkv = (size_t)(m.H + 2 * m.H_kv) * m.D;
+  const size_t wide = (size_t)m.d > (size_t)m.H * m.D ? m.d : (size_t)m.H * m.D;
+  Buffers t{};
+  t.x = (float*)take(R * m.d * 4);
+  t.xn = (bf16*)take(R * wide * 2);
+  t.qkv = (float*)take(R * nqkv * 4);
+  t.q = (bf16*)take(R * m.H * m.D * 2);
+  t.att = (bf16*)take(R * m.H * m.D * 2);
+  t.tmp = (float*)take(R * (size_t)(m.F > m.d ? m.F : m.d) * 4);
+  t.tmp2 = (float*)take(R * (size_t)m.F * 4);
+  t.hf = (bf16*)take(R * (size_t)m.F * 2);
+  t.logits = (float*)take(R * (size_t)m.V * 4);
+  t.sel_id = (int32_t*)take(R * BITA_MAX_TOPK * 4);
+  t.sel_val = (float*)take(R * BITA_MAX_TOPK * 4);
+  t.pos = (int32_t*)take(R * 4);
+  t.row_token = (int32_t*)take(R * 4);
+  const size_t S = attn_splits(m.H, 1);
+  t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
+  t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
+  t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
+  t.state = (DevState*)take(sizeof(DevState));
+  t.rec = (DevRecord*)take(sizeof(DevRecord));
+  t.plan_step = take(PLAN_REGION_BYTES);
+  t.plan_prefill = take(PLAN_REGION_BYTES);
+  t.query_tokens = (int32_t*)take(PREFILL_CHUNK * 4);
+  t.tree_in = (int32_t*)take(BITA_MAX_NODES * 4);
+  if (b) *b = t;
+  return off;
+}
+
+}  // namespace
+
+struct bita_ctx {
+  bita_model_dims m;
+  int n_mask;
+  std::vector<const void*> wqkv, wo, wg, wu, wd, g_attn, g_ffn, prompt_k, prompt_v;
+  const void *tok_emb, *mask_emb, *g_final, *lm_head;
+  cudaStream_t stream;
+  Buffers b;
+  HostPlan step_plan, prefill_plan;
+  DevRecord* rec_host;      // pinned
+  int len_upper;            // upper bound of the device-side cache length
+  bool prefilled;
+  float* dbg;
+  int launches;
+};
+
+namespace {
+
+void gemm(bita_ctx* c, const bf16* X, const void* W, float* Y, int M, int N, int K) {
+  k_gemm_simple<<<(N + 3) / 4, 128, 0, c->stream>>>(X, (const bf16*)W, Y, M, N, K, N);
+  c->launches++;
+}
+
+void launch_attention(const AttnArgs& a, cudaStream_t s) {
+  dim3 g1(a.H, a.S, a.B), g2(a.M, a.H, a.B);
+  if (a.D == 128) {
+    k_attn_simple<128><<<g1, 128, 0, s>>>(a);
+    k_attn_merge<128><<<g2, 128, 0, s>>>(a);
+  } else {
+    k_attn_simple<64><<<g1, 128, 0, s>>>(a);
+    k_attn_merge<64><<<g2, 64, 0, s>>>(a);
+  }
+}
+
+// The layer stack over one packed block, then (optionally) the LM head and selection.
+int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_dev, bool want_logits) {
+  const bita_model_dims& m = c->m;
+  const DevPlan& P = hp.dev;
+  const int M = P.M;
+  cudaStream_t s = c->stream;
+  Buffers& b = c->b;
+  const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
+  k_embed<<<M, 256, 0, s>>>(P, b.state, tree_dev, b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb,
+                            m.d, m.V, b.x, b.pos, b.row_token);
+  c->launches++;
+  const int nqkv = (m.H + 2 * m.H_kv) * m.D;
+  for (int l = 0; l < m.L; ++l) {
+    bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
+    bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
+    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_attn[l], m.d, m.rms_eps, b.xn);
+    gemm(c, b.xn, c->wqkv[l], b.qkv, M, nqkv, m.d);
+    k_rope_kv<<<M, 256, 0, s>>>(b.qkv, b.pos, b.rope_tab, b.state, m.H, m.H_kv, m.D, kv->C_max, b.q, kc, vc);
+    AttnArgs a{};
+    a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
+    a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
+    a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
+    a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
+    a.S = attn_splits(m.H, 1); a.scale = 1.0f / sqrtf((float)m.D);
+    launch_attention(a, s);
+    gemm(c, b.att, c->wo[l], b.tmp, M, m.d, m.H * m.D);
+    k_add<<<(unsigned)(((size_t)M * m.d + 255) / 256), 256, 0, s>>>(b.x, b.tmp, (size_t)M * m.d);
+    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn);
+    gemm(c, b.xn, c->wg[l], b.tmp, M, m.F, m.d);
+    gemm(c, b.xn, c->wu[l], b.tmp2, M, m.F, m.d);
+    k_swiglu<<<(unsigned)(((size_t)M * m.F + 255) / 256), 256, 0, s>>>(b.tmp, b.tmp2, (size_t)M * m.F, b.hf);
+    gemm(c, b.hf, c->wd[l], b.tmp, M, m.d, m.F);
+    k_add<<<(unsigned)(((size_t)M * m.d + 255) / 256), 256, 0, s>>>(b.x, b.tmp, (size_t)M * m.d);
+    c->launches += 8;
+    if (c->dbg)
+      CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)l * BITA_MAX_ROWS * m.d, b.x, (size_t)M * m.d * 4,
+                             cudaMemcpyDeviceToDevice, s));
+  }
+  if (want_logits) {
+    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_final, m.d, m.rms_eps, b.xn);
+    gemm(c, b.xn, c->lm_head, b.logits, M, m.V, m.d);
+    k_select<<<M, 256, 0, s>>>(P, b.logits, m.V, b.sel_id, b.sel_val);
+    c->launches += 2;
+    if (c->dbg)
+      CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,
+                             cudaMemcpyDeviceToDevice, s));
+  }
+  CU_TRY(cudaGetLastError());
+  return BITA_OK;
+}
+
+void fill_out(const DevRecord* r, bita_step_out* out) {
+  out->status = r->status;
+  out->n_out = r->n_out;
+  out->new_len = r->new_len;
+  memcpy(out->out_tokens, r->out_tokens, sizeof(out->out_tokens));
+  memcpy(out->accepted_idx, r->accepted_idx, sizeof(out->accepted_idx));
+  memcpy(out->next_tree, r->next_tree, sizeof(out->next_tree));
+}
+
+}  // namespace
+
+extern "C" {
+
+int bita_workspace_bytes(const bita_model_dims* dims, const bita_tree_template* tmpl, int n_mask, size_t* out_bytes) {
+  if (!out_bytes) return BITA_ERR_INVALID_ARG;
+  int rc = check_dims(dims);
+  if (rc) return rc;
+  HostPlan p;
+  rc = build_step_plan(tmpl, n_mask, &p);
+  if (rc) return rc;
+  *out_bytes = carve(*dims, nullptr, nullptr);
+  return BITA_OK;
+}
+
+int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w, const bita_tree_template* tmpl,
+              int n_mask, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!out || !w || !workspace) return BITA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_dims(dims);
+  if (rc) return rc;
+  if (!w->tok_emb || !w->g_final || !w->lm_head || !w->wqkv || !w->wo || !w->wg || !w->wu || !w->wd || !w->g_attn ||
+      !w->g_ffn)
+    return BITA_ERR_INVALID_ARG;
+  if (n_mask > 0 && !w->mask_emb) return BITA_ERR_INVALID_ARG;
+  if (dims->P > 0 && (!w->prompt_k || !w->prompt_v)) return BITA_ERR_INVALID_ARG;
+  bita_ctx* c = new (std::nothrow) bita_ctx();
+  if (!c) return BITA_ERR_INVALID_ARG;
+  rc = build_step_plan(tmpl, n_mask, &c->step_plan);
+  if (rc) { delete c; return rc; }
+  if (((uintptr_t)workspace % ALIGN) || workspace_bytes < carve(*dims, nullptr, nullptr)) {
+    delete c;
+    return BITA_ERR_WORKSPACE;
+  }
+  c->m = *dims;
+  c->n_mask = n_mask;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->tok_emb = w->tok_emb; c->mask_emb = w->mask_emb; c->g_final = w->g_final; c->lm_head = w->lm_head;
+  const int L = dims->L;
+  auto cp = [&](std::vector<const void*>& v, const void* const* src, bool need) -> bool {
+    v.assign(L, nullptr);
+    if (!src) return !need;
+    for (int l = 0; l < L; ++l) { v[l] = src[l]; if (need && !src[l]) return false; }
+    return true;
+  };
+  bool ok = cp(c->wqkv, w->wqkv, true) && cp(c->wo, w->wo, true) && cp(c->wg, w->wg, true) && cp(c->wu, w->wu, true) &&
+            cp(c->wd, w->wd, true) && cp(c->g_attn, w->g_attn, true) && cp(c->g_ffn, w->g_ffn, true) &&
+            cp(c->prompt_k, w->prompt_k, dims->P > 0) && cp(c->prompt_v, w->prompt_v, dims->P > 0);
+  if (!ok) { delete c; return BITA_ERR_INVALID_ARG; }
+  carve(*dims, (uint8_t*)workspace, &c->b);
+  c->rec_host = nullptr;
+  c->dbg = nullptr;
+  c->launches = 0;
+  c->prefilled = false;
+  c->len_upper = 0;
+  auto fail = [&](int code) { if (c->rec_host) cudaFreeHost(c->rec_host); delete c; return code; };
+  if (cudaMallocHost((void**)&c->rec_host, sizeof(DevRecord)) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  memset(c->rec_host, 0, sizeof(DevRecord));
+  // rotary table in double precision: angle = pos * theta^(-2j/D)
+  {
+    const int half = dims->D / 2, npos = dims->C_max + 64;
+    std::vector<float2> tab((size_t)npos * half);
+    std::vector<double> inv(half);
+    for (int j = 0; j < half; ++j) inv[j] = pow((double)dims->rope_theta, -2.0 * j / dims->D);
+    for (int p = 0; p < npos; ++p)
+      for (int j = 0; j < half; ++j) {
+        const double ang = (double)p * inv[j];
+        tab[(size_t)p * half + j] = make_float2((float)cos(ang), (float)sin(ang));
+      }
+    if (cudaMemcpyAsync(c->b.rope_tab, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, c->stream) !=
+            cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+      return fail(BITA_ERR_CUDA);
+  }
+  rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
+  if (rc) return fail(rc);
+  k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  *out = c;
+  return BITA_OK;
+}
+
+int bita_reset(bita_ctx* c, bita_kv* kv) {
+  if (!c || !kv) return BITA_ERR_INVALID_ARG;
+  k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  c->prefilled = false;
+  c->len_upper = 0;
+  return BITA_OK;
+}
+
+int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count, bita_step_out* out) {
+  if (!c || !kv || !kv->k || !kv->v || !tokens || count < 1) return BITA_ERR_INVALID_ARG;
+  if (kv->C_max != c->m.C_max) return BITA_ERR_INVALID_ARG;
+  for (int i = 0; i < count; ++i)
+    if (tokens[i] < 0 || tokens[i] >= c->m.V) return BITA_ERR_INVALID_ARG;
+  if ((long)c->len_upper + count + c->n_mask > kv->C_max) return BITA_ERR_KV_FULL;
+  c->launches = 0;
+  for (int done = 0; done < count;) {
+    const int cnt = count - done < PREFILL_CHUNK ? count - done : PREFILL_CHUNK;
+    const bool last = done + cnt == count;
+    build_prefill_plan(cnt, c->n_mask, last, c->step_plan.k_max, &c->prefill_plan);
+    int rc = upload_plan(&c->prefill_plan, c->b.plan_prefill, c->stream);
+    if (rc) return rc;
+    CU_TRY(cudaMemcpyAsync(c->b.query_tokens, tokens + done, cnt * 4, cudaMemcpyHostToDevice, c->stream));
+    rc = run_block(c, kv, c->prefill_plan, nullptr, last);
+    if (rc) return rc;
+    k_prefill_finish<<<1, 32, 0, c->stream>>>(c->prefill_plan.dev, c->step_plan.dev, c->b.state, c->b.sel_id, c->b.rec,
+                                              last ? 1 : 0);
+    c->launches++;
+    CU_TRY(cudaStreamSynchronize(c->stream));   // the plan region and token buffer are reused by the next chunk
+    done += cnt;
+  }
+  CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  c->len_upper = c->rec_host->new_len;
+  c->prefilled = true;
+  if (out) fill_out(c->rec_host, out);
+  return c->rec_host->status ? BITA_ERR_TIMEOUT : BITA_OK;
+}
+
+int bita_step_enqueue(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens_dev) {
+  if (!c || !kv || !kv->k || !kv->v) return BITA_ERR_INVALID_ARG;
+  if (kv->C_max != c->m.C_max) return BITA_ERR_INVALID_ARG;
+  if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
+  if ((long)c->len_upper + c->step_plan.M > kv->C_max) return BITA_ERR_KV_FULL;
+  c->launches = 0;
+  int rc = run_block(c, kv, c->step_plan, tree_tokens_dev, true);
+  if (rc) return rc;
+  k_accept<<<1, 32, 0, c->stream>>>(c->step_plan.dev, c->b.state, c->b.row_token, c->b.sel_id, c->b.rec);
+  k_compact<<<c->m.L * c->m.H_kv, 64, 0, c->stream>>>(c->b.rec, c->m.D, kv->C_max, (bf16*)kv->k, (bf16*)kv->v);
+  c->launches += 2;
+  CU_TRY(cudaGetLastError());
+  CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
+  c->len_upper += c->step_plan.max_depth + 1;
+  return BITA_OK;
+}
+
+int bita_step_finish(bita_ctx* c, bita_step_out* out) {
+  if (!c || !out) return BITA_ERR_INVALID_ARG;
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  c->len_upper = c->rec_host->new_len;
+  fill_out(c->rec_host, out);
+  return c->rec_host->status ? BITA_ERR_TIMEOUT : BITA_OK;
+}
+
+int bita_step(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens, bita_step_out* out) {
+  if (!c || !out) return BITA_ERR_INVALID_ARG;
+  const int32_t* dev = nullptr;
+  if (tree_tokens && c->step_plan.N > 0) {
+    for (int i = 0; i < c->step_plan.N; ++i)
+      if (tree_tokens[i] < -1 || tree_tokens[i] >= c->m.V) return BITA_ERR_INVALID_ARG;
+    if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
+    CU_TRY(cudaMemcpyAsync(c->b.tree_in, tree_tokens, c->step_plan.N * 4, cudaMemcpyHostToDevice, c->stream));
+    dev = c->b.tree_in;
+  }
+  int rc = bita_step_enqueue(c, kv, dev);
+  if (rc) return rc;
+  return bita_step_finish(c, out);
+}
+
+int bita_set_debug_buffer(bita_ctx* c, void* dev_buf, size_t bytes) {
+  if (!c) return BITA_ERR_INVALID_ARG;
+  if (dev_buf) {
+    const size_t need = ((size_t)c->m.L * BITA_MAX_ROWS * c->m.d + (size_t)BITA_MAX_ROWS * c->m.V) * 4;
+    if (bytes < need) return BITA_ERR_WORKSPACE;
+  }
+  c->dbg = (float*)dev_buf;
+  return BITA_OK;
+}
+
+int bita_block_rows(const bita_ctx* c) { return c ? c->step_plan.M : BITA_ERR_INVALID_ARG; }
+int bita_last_launch_count(const bita_ctx* c) { return c ? c->launches : BITA_ERR_INVALID_ARG; }
+
+void bita_destroy(bita_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  if (c->rec_host) cudaFreeHost(c->rec_host);
+  delete c;
+}
+
+const char* bita_strerror(int code) {
+  switch (code) {
+    case BITA_OK: return "ok";
+    case BITA_ERR_INVALID_ARG: return "invalid argument";
+    case BITA_ERR_BAD_TEMPLATE: return "bad tree template";
+    case BITA_ERR_KV_FULL: return "KV cache full";
+    case BITA_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case BITA_ERR_CUDA: return "CUDA runtime error";
+    case BITA_ERR_TIMEOUT: return "device-side wait timed out";
+    case BITA_ERR_NOT_PREFILLED: return "bita_prefill has not been called";
+    default: return "unknown error";
+  }
+}
+
+int bita_last_cuda_error(void) { return g_last_cuda_error; }
+
+int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes) {
+  if (!out_bytes || M < 1 || M > BITA_MAX_ROWS || N < 1 || K < 8 || K % 8) return BITA_ERR_INVALID_ARG;
+  *out_bytes = ALIGN;
+  return BITA_OK;
+}
+
+int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, int32_t K, void* workspace,
+                   size_t workspace_bytes, void* cuda_stream) {
+  size_t need = 0;
+  int rc = bita_gemm_workspace_bytes(M, N, K, &need);
+  if (rc) return rc;
+  if (!X || !W || !Y) return BITA_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < need) return BITA_ERR_WORKSPACE;
+  k_gemm_simple<<<(N + 3) / 4, 128, 0, (cudaStream_t)cuda_stream>>>((const bf16*)X, (const bf16*)W, (float*)Y, M, N, K, N);
+  CU_TRY(cudaGetLastError());
+  return BITA_OK;
+}
+
+int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
+  if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
+  const size_t S = attn_splits(H, B);
+  *out_bytes = align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
+  return BITA_OK;
+}
+
+int bita_tree_attention(const void* q, const void* k, const void* v, const uint32_t* vis, const void* prompt_k,
+                        const void* prompt_v, const uint8_t* sees_prompt, const int32_t* ctx_len, void* out, int32_t B,
+                        int32_t M, int32_t H, int32_t H_kv, int32_t D, int32_t P, int32_t C_max, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+  size_t need = 0;
+  int rc = bita_attention_workspace_bytes(B, M, H, D, &need);
+  if (rc) return rc;
+  if (!q || !k || !v || !vis || !ctx_len || !out || H_kv < 1 || H % H_kv || P < 0 || P > 64 || C_max < M)
+    return BITA_ERR_INVALID_ARG;
+  if (P > 0 && (!prompt_k || !prompt_v || !sees_prompt)) return BITA_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace % ALIGN)) return BITA_ERR_WORKSPACE;
+  AttnArgs a{};
+  const int W = (M + 31) / 32;
+  a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
+  a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
+  a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
+  a.S = attn_splits(H, B);
+  a.part_ml = (float*)workspace;
+  a.part_acc = (float*)((uint8_t*)workspace + align_up((size_t)B * H * a.S * M * 2 * 4));
+  a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
+  a.scale = 1.0f / sqrtf((float)D);
+  launch_attention(a, (cudaStream_t)cuda_stream);
+  CU_TRY(cudaGetLastError());
+  return BITA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,302 @@
+// Element-wise and integer kernels of one decoding pass: embedding/packing, RMSNorm,
+// rotary embedding + cache write, SwiGLU, argmax/top-k selection, the greedy
+// verification walk, next-tree construction and cache compaction.
+#pragma once
+
+#include "common.cuh"
+
+namespace bita {
+
+// ---------------------------------------------------------------------------------------------
+// Packing (Sec. 3.2 "flatten the draft candidate token tree, along with the attached mask
+// tokens"; Appendix B): row 0 = last accepted token, rows 1..N = tree tokens (token -1 -> zero
+// row), then the mask embeddings.  Position ids: C + rel_pos.
+// x: fp32 [M][d] residual stream; pos: int32 [M].
+__global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int32_t* __restrict__ tree_tokens,
+                        const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
+                        const bf16* __restrict__ mask_emb, int d, int V, float* __restrict__ x,
+                        int32_t* __restrict__ pos, int32_t* __restrict__ row_token) {
+  const int r = blockIdx.x;
+  const int kind = plan.row_kind[r];
+  const int idx = plan.row_idx[r];
+  const bf16* src = nullptr;
+  int tok = -1;
+  if (kind == ROW_ROOT) tok = st->root;
+  else if (kind == ROW_NODE) tok = tree_tokens ? tree_tokens[idx] : st->tree[idx];
+  else if (kind == ROW_QUERY) tok = query_tokens[idx];
+  if (kind == ROW_MASK) src = mask_emb + (size_t)idx * d;
+  else if (tok >= 0 && tok < V) src = tok_emb + (size_t)tok * d;
+  if (threadIdx.x == 0) {
+    pos[r] = st->len + plan.rel_pos[r];
+    row_token[r] = (tok >= 0 && tok < V) ? tok : -1;
+  }
+  float* xr = x + (size_t)r * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) xr[c] = src ? bf2f(src[c]) : 0.0f;
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm: xn = x * g / sqrt(mean(x^2) + eps), fp32 in, bf16 out.  One block per row.
+__global__ void k_rmsnorm(const float* __restrict__ x, const bf16* __restrict__ g, int d, float eps,
+                          bf16* __restrict__ xn) {
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const float* xr = x + (size_t)r * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) { float v = xr[c]; ss += v * v; }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
+  }
+  __syncthreads();
+  const float inv = red[0];
+  bf16* o = xn + (size_t)r * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rotary embedding (half-split pairing: dims j and j + D/2) at the row's position id, then
+// q -> bf16 [M][H][D], k/v -> cache slot C + r of layout [H_kv][C_max][D].
+// rope_tab: float2 (cos, sin) [positions][D/2], computed in double on the host.
+__global__ void k_rope_kv(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
+                          const float2* __restrict__ rope_tab, const DevState* __restrict__ st, int H, int H_kv,
+                          int D, int C_max, bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc) {
+  const int r = blockIdx.x;
+  const int half = D >> 1;
+  const int p = pos[r];
+  const int slot = st->len + r;
+  const int nq = H * half, nk = H_kv * half;
+  const float* row = qkv + (size_t)r * (H + 2 * H_kv) * D;
+  for (int t = threadIdx.x; t < nq + nk; t += blockDim.x) {
+    const bool isq = t < nq;
+    const int u = isq ? t : t - nq;
+    const int h = u / half, j = u - h * half;
+    const float* src = row + (isq ? 0 : H * D) + h * D;
+    const float2 cs = rope_tab[(size_t)p * half + j];
+    const float a = src[j], b = src[j + half];
+    const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
+    if (isq) {
+      bf16* dst = q + ((size_t)r * H + h) * D;
+      dst[j] = f2bf(ra);
+      dst[j + half] = f2bf(rb);
+    } else if (slot < C_max) {
+      bf16* dst = kc + ((size_t)h * C_max + slot) * D;
+      dst[j] = f2bf(ra);
+      dst[j + half] = f2bf(rb);
+    }
+  }
+  if (slot < C_max) {
+    const float* vsrc = row + (H + H_kv) * D;
+    for (int t = threadIdx.x; t < H_kv * D; t += blockDim.x) {
+      const int h = t / D, j = t - h * D;
+      vc[((size_t)h * C_max + slot) * D + j] = f2bf(vsrc[t]);
+    }
+  }
+}
+
+// x += t (residual), fp32.
+__global__ void k_add(float* __restrict__ x, const float* __restrict__ t, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) x[i] += t[i];
+}
+
+// hf = silu(gate) * up -> bf16.  gate/up fp32 [M][F].
+__global__ void k_swiglu(const float* __restrict__ gate, const float* __restrict__ up, size_t n,
+                         bf16* __restrict__ hf) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    const float g = gate[i];
+    hf[i] = f2bf(g / (1.0f + __expf(-g)) * up[i]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Argmax / sorted top-k of each logits row, order = (value descending, token id ascending).
+// One block per row; pass t picks the best entry strictly after the previous pick.
+// sel_id: int32 [M][BITA_MAX_TOPK], sel_val: fp32 [M][BITA_MAX_TOPK].
+__device__ __forceinline__ bool before(float v1, int i1, float v2, int i2) {
+  return v1 > v2 || (v1 == v2 && i1 < i2);
+}
+
+__global__ void k_select(DevPlan plan, const float* __restrict__ logits, int V, int32_t* __restrict__ sel_id,
+                         float* __restrict__ sel_val) {
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  __shared__ float pv;
+  __shared__ int pi;
+  const int r = blockIdx.x;
+  const int kind = plan.row_kind[r];
+  const int K = (kind == ROW_MASK) ? plan.k_max : 1;
+  const float* row = logits + (size_t)r * V;
+  float prev_v = 0.f;
+  int prev_i = -1;
+  for (int t = 0; t < K; ++t) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int c = threadIdx.x; c < V; c += blockDim.x) {
+      const float v = row[c];
+      if (!(v == v)) continue;
+      if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;  // not strictly after the previous pick
+      if (before(v, c, bv, bi)) { bv = v; bi = c; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int nw = blockDim.x >> 5;
+      bv = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+      bi = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      if (threadIdx.x == 0) {
+        pv = bv;
+        pi = (bi == 0x7fffffff) ? -1 : bi;
+        sel_id[(size_t)r * BITA_MAX_TOPK + t] = pi;
+        sel_val[(size_t)r * BITA_MAX_TOPK + t] = bv;
+      }
+    }
+    __syncthreads();
+    prev_v = pv;
+    prev_i = pi;
+    if (prev_i < 0) break;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Greedy verification (Algorithm 1, else-branch, general-tree form) and next-tree construction
+// (Algorithm 1, "Get C^t by selecting the top k predictions ... of the mask token group linked to
+// the last accepted candidate token").  One warp: lanes scan the children of the current node.
+__global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t* __restrict__ row_token,
+                         const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec) {
+  const int lane = threadIdx.x;
+  const int N = plan.N;
+  int cur = -1;
+  int a = sel_id[0];
+  int n_acc = 0;
+  for (int round = 0; round < BITA_MAX_DEPTH; ++round) {
+    int found = 0x7fffffff;
+    for (int x = lane; x < N; x += 32) {
+      const int tok = row_token[1 + x];
+      if (plan.parent[x] == cur && tok >= 0 && tok == a) { found = x; break; }   // lowest index first
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+    if (found == 0x7fffffff) break;
+    if (lane == 0) { rec->accepted_idx[n_acc] = found; rec->out_tokens[n_acc] = a; }
+    ++n_acc;
+    cur = found;
+    a = sel_id[(size_t)(1 + cur) * BITA_MAX_TOPK];
+  }
+  // group attached to the last accepted node, else to its nearest ancestor that has one
+  int at = cur, shift = 0, g = -1;
+  while (true) {
+    g = plan.group_of[at + 1];
+    if (g >= 0 || at < 0) break;
+    at = plan.parent[at];
+    ++shift;
+  }
+  const int C = st->len;
+  __syncwarp();
+  for (int x = lane; x < N; x += 32) {
+    const int m = plan.depth[x] - 1 + shift;
+    int tok = -1;
+    if (g >= 0 && m < plan.n_mask) {
+      const int mrow = 1 + N + g * plan.n_mask + m;
+      tok = sel_id[(size_t)mrow * BITA_MAX_TOPK + plan.rank[x]];
+    }
+    rec->next_tree[x] = tok;
+    st->tree[x] = tok;
+  }
+  for (int x = N + lane; x < BITA_MAX_NODES; x += 32) rec->next_tree[x] = -1;
+  if (lane == 0) {
+    rec->out_tokens[n_acc] = a;
+    for (int j = n_acc + 1; j <= BITA_MAX_DEPTH; ++j) rec->out_tokens[j] = -1;
+    for (int j = n_acc; j < BITA_MAX_DEPTH; ++j) rec->accepted_idx[j] = -1;
+    rec->n_out = n_acc + 1;
+    rec->n_acc = n_acc;
+    rec->old_len = C;
+    rec->new_len = C + 1 + n_acc;
+    rec->status = st->status;
+    st->len = C + 1 + n_acc;
+    st->root = a;
+  }
+}
+
+// First pass (Algorithm 1, t = 1): the last query row's argmax is emitted, the one mask group that
+// follows it drafts the first tree.  `last` = this is the final chunk of the query.
+__global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __restrict__ st,
+                                 const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec, int last) {
+  const int lane = threadIdx.x;
+  const int C = st->len;
+  const int T = chunk.n_query;
+  __syncwarp();
+  if (last) {
+    const int a = sel_id[(size_t)(T - 1) * BITA_MAX_TOPK];
+    const int N = step_plan.N;
+    for (int x = lane; x < N; x += 32) {
+      const int m = step_plan.depth[x] - 1;
+      int tok = -1;
+      if (m < chunk.n_mask) tok = sel_id[(size_t)(T + m) * BITA_MAX_TOPK + step_plan.rank[x]];
+      rec->next_tree[x] = tok;
+      st->tree[x] = tok;
+    }
+    for (int x = N + lane; x < BITA_MAX_NODES; x += 32) rec->next_tree[x] = -1;
+    if (lane == 0) {
+      rec->out_tokens[0] = a;
+      for (int j = 1; j <= BITA_MAX_DEPTH; ++j) rec->out_tokens[j] = -1;
+      for (int j = 0; j < BITA_MAX_DEPTH; ++j) rec->accepted_idx[j] = -1;
+      rec->n_out = 1;
+      rec->n_acc = 0;
+      rec->old_len = C;
+      rec->new_len = C + T;
+      rec->status = st->status;
+      st->root = a;
+    }
+  }
+  if (lane == 0) st->len = C + T;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Cache compaction ("its prediction, along with its subsequent tokens, is discarded", Fig. 3
+// caption): the j-th accepted node's entry moves from slot C+1+idx_j to slot C+1+j.  One thread
+// owns a 16-byte column chunk and walks j upwards, which is alias-safe because idx_j >= j and
+// idx is increasing along a path.  grid = (L * H_kv), cache layout [L][H_kv][C_max][D].
+__global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, bf16* __restrict__ kc,
+                          bf16* __restrict__ vc) {
+  const int n_acc = rec->n_acc;
+  if (n_acc == 0) return;
+  const int C = rec->old_len;
+  const int chunks = D / 8;                       // 16-byte chunks per row
+  const size_t base = (size_t)blockIdx.x * C_max * D;
+  for (int t = threadIdx.x; t < 2 * chunks; t += blockDim.x) {
+    bf16* buf = (t < chunks ? kc : vc) + base;
+    const int c = (t < chunks ? t : t - chunks) * 8;
+    for (int j = 0; j < n_acc; ++j) {
+      const int src = C + 1 + rec->accepted_idx[j];
+      const int dst = C + 1 + j;
+      if (src != dst && src < C_max) {
+        const uint4 v = *reinterpret_cast<const uint4*>(buf + (size_t)src * D + c);
+        *reinterpret_cast<uint4*>(buf + (size_t)dst * D + c) = v;
+      }
+    }
+  }
+}
+
+__global__ void k_reset_state(DevState* st) {
+  if (threadIdx.x == 0) { st->len = 0; st->root = -1; st->status = 0; st->pad = 0; }
+  for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
+}
+
+}  // namespace bita
