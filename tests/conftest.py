@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+    # the C-ABI library is built in-tree (nvcc cross-compiles without a GPU)
+    from paper_2401_12522_b200.build import build
+    build()
 
 
 def pytest_collection_modifyitems(config, items):

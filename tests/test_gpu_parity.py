@@ -1,0 +1,204 @@
+"""CUDA library against the CPU oracle on the same seeded inputs (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from helpers import MICRO, block_for, oracle_model, orc, prompt_tokens
+from lockstep import HIDDEN_REL_L2, LOGIT_TOL_RMS, Lockstep, rel_l2, run_lockstep
+
+pytestmark = pytest.mark.gpu
+
+
+def test_generators_are_bit_identical_on_cpu_and_gpu():
+    for seed, stream, shape in [(1, 2, (1000, 37)), (0x5EED0001, 117, (4096, 64))]:
+        a = synth.pseudo_normal(seed, stream, shape, 0.02, dtype=torch.bfloat16, device="cpu")
+        b = synth.pseudo_normal(seed, stream, shape, 0.02, dtype=torch.bfloat16, device="cuda:0")
+        assert torch.equal(a, b.cpu())
+
+
+# ------------------------------------------------------------------ single operators
+
+@pytest.mark.parametrize("M,N,K", [(1, 128, 64), (19, 1376, 256), (19, 256, 688), (69, 1000, 4096),
+                                   (133, 384, 1024), (256, 130, 520)])
+def test_projection_matches_fp64_matmul(M, N, K):
+    from paper_2401_12522_b200 import bita_gemm_bf16
+    X = synth.pseudo_normal(3, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda:0")
+    W = synth.pseudo_normal(3, 2, (N, K), 0.02, dtype=torch.bfloat16, device="cuda:0")
+    Y = bita_gemm_bf16(X, W).cpu().numpy().astype(np.float64)
+    ref = X.cpu().double().numpy() @ W.cpu().double().numpy().T
+    # fp32 accumulation of exact bf16 products: error ~ sqrt(K) * 2^-24 relative to the row scale
+    assert rel_l2(Y, ref) < 1e-5
+    assert np.abs(Y - ref).max() <= 1e-4 * np.abs(ref).max()
+
+
+def _random_attention_case(seed, B, M, H, H_kv, D, P, C, tmpl):
+    dev = "cuda:0"
+    C_max = C + M + 3
+    q = synth.pseudo_normal(seed, 1, (B, M, H, D), 1.0, dtype=torch.bfloat16, device=dev)
+    k = synth.pseudo_normal(seed, 2, (B, H_kv, C_max, D), 1.0, dtype=torch.bfloat16, device=dev)
+    v = synth.pseudo_normal(seed, 3, (B, H_kv, C_max, D), 1.0, dtype=torch.bfloat16, device=dev)
+    pk = synth.pseudo_normal(seed, 4, (H_kv, max(P, 1), D), 1.0, dtype=torch.bfloat16, device=dev)
+    pv = synth.pseudo_normal(seed, 5, (H_kv, max(P, 1), D), 1.0, dtype=torch.bfloat16, device=dev)
+    blk = block_for(tmpl, 4)
+    assert blk.M == M
+    W = (M + 31) // 32
+    vis = np.zeros((M, W), dtype=np.uint32)
+    for r in range(M):
+        for c in np.nonzero(blk.vis[r])[0]:
+            vis[r, c >> 5] |= np.uint32(1 << (c & 31))
+    vis_t = torch.from_numpy(np.broadcast_to(vis.view(np.int32), (B, M, W)).copy()).to(dev)
+    sp = torch.from_numpy(np.broadcast_to(blk.sees_prompt.astype(np.uint8), (B, M)).copy()).to(dev)
+    ctx = torch.tensor([C - (b % 3) for b in range(B)], dtype=torch.int32, device=dev)
+    return q, k, v, pk, pv, vis_t, sp, ctx, blk
+
+
+@pytest.mark.parametrize("B,N,H,H_kv,D,P,C", [(1, 16, 4, 4, 64, 16, 70), (2, 16, 8, 2, 128, 16, 300),
+                                              (1, 64, 4, 4, 128, 0, 513), (1, 128, 2, 1, 128, 5, 40),
+                                              (1, 0, 4, 2, 64, 16, 0)])
+def test_tree_attention_matches_oracle(B, N, H, H_kv, D, P, C):
+    from paper_2401_12522_b200 import bita_tree_attention
+    tmpl = synth.random_recursive_template(N + 1, N) if N else synth.empty_template()
+    M = 1 + N + 4
+    q, k, v, pk, pv, vis, sp, ctx, blk = _random_attention_case(7, B, M, H, H_kv, D, P, C, tmpl)
+    out = bita_tree_attention(q, k, v, vis, pk if P else None, pv if P else None, sp if P else None, ctx,
+                              H_kv=H_kv, P=P)
+    m = orc.Model(L=1, d=H * D, H=H, H_kv=H_kv, D=D, F=8, V=8, P=P, n_mask=4, rms_eps=1e-5, rope_theta=1e4,
+                  weights={})
+    for b in range(B):
+        Cb = int(ctx[b])
+        keys = k[b].double().cpu().numpy()[:, : Cb + M]
+        vals = v[b].double().cpu().numpy()[:, : Cb + M]
+        allowed = np.concatenate([np.ones((M, Cb), dtype=bool), blk.vis], axis=1)
+        if P:
+            keys = np.concatenate([keys, pk.double().cpu().numpy()], axis=1)
+            vals = np.concatenate([vals, pv.double().cpu().numpy()], axis=1)
+            allowed = np.concatenate([allowed, np.repeat(blk.sees_prompt[:, None], P, axis=1)], axis=1)
+        ref = orc._attention(m, q[b].double().cpu().numpy(), keys, vals, allowed)
+        got = out[b].float().cpu().numpy().astype(np.float64)
+        assert rel_l2(got, ref) < 6e-3            # output is rounded to bf16 (2^-9 relative per element)
+        assert np.abs(got - ref).max() < 3e-2
+
+
+# ------------------------------------------------------------------ the whole pass, lockstep
+
+def test_tiny_config_lockstep_32_steps():
+    shape = synth.CONFIGS["tiny"]
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    ls = run_lockstep(shape, 0x5EED0001, tmpl, shape.steps)
+    assert ls.exact + ls.adopted == shape.steps + 1
+    assert ls.exact >= (shape.steps + 1) // 2      # most passes have clear margins
+    print(f"tiny lockstep: exact={ls.exact} adopted={ls.adopted} hidden={ls.max_hidden:.2e} "
+          f"logits={ls.max_logit:.2e}xRMS")
+    ls.close()
+
+
+TEMPLATES = {
+    "comb-n3k5-pernode": (lambda: synth.comb_template(3, 5), 3),
+    "comb-n4k3-pernode": (lambda: synth.comb_template(4, 3), 4),
+    "chain": (lambda: synth.chain_template(3), 3),
+    "empty": (lambda: synth.empty_template(), 3),
+    "product-pernode": (lambda: synth.product_rule_template((3, 3, 3), (3, 3, 3), per_node_groups=True), 3),
+    "random-40": (lambda: synth.random_recursive_template(4, 40, max_depth=6), 3),
+}
+
+
+@pytest.mark.parametrize("name", sorted(TEMPLATES))
+def test_templates_lockstep_with_planted_paths(name):
+    from dataclasses import replace
+    mk, n_mask = TEMPLATES[name]
+    shape = replace(synth.CONFIGS["tiny"], n_mask=n_mask)
+    tmpl = mk()
+    seed = 0x5EED0002
+    prompt = prompt_tokens(seed, 37, shape.V)
+    # the true continuation, from the oracle's definition of the output
+    model = oracle_model(shape, seed)
+    ref = orc.ar_greedy(model, prompt, 40)
+
+    def tree_fn(step, ls):
+        if step % 3 == 0:
+            return None                                        # the model's own drafts
+        done = ls.st.C - len(prompt) + 1
+        base = list(ls.st.tree)
+        return synth.plant_tree(tmpl, base, ref[done: done + 8], seed, step, 0.8, shape.V)
+
+    ls = run_lockstep(shape, seed, tmpl, 10, prompt=prompt, tree_fn=tree_fn)
+    n = min(len(ls.emitted), len(ref))
+    if ls.adopted == 0:
+        assert ls.emitted[:n] == ref[:n]                       # lossless: equals greedy AR decoding
+    ls.close()
+
+
+def test_gpu_generation_is_lossless_against_its_own_autoregressive_run():
+    """BiTA loop and one-token-per-pass loop of the library emit the same tokens (up to sub-tolerance ties)."""
+    from paper_2401_12522_b200 import Bita
+    shape = synth.CONFIGS["tiny"]
+    seed = 0x5EED0003
+    w = synth.make_weights(shape, seed, dtype=torch.bfloat16, device="cuda:0")
+    prompt = prompt_tokens(seed, shape.prompt_len, shape.V)
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    n_new = 48
+    ar = Bita(shape, w, synth.empty_template(), C_max=512)
+    seq_ar = list(ar.prefill(prompt)["out_tokens"])
+    while len(seq_ar) < n_new:
+        seq_ar += ar.step()["out_tokens"]
+    ar.close()
+    bt = Bita(shape, w, tmpl, C_max=512)
+    seq = list(bt.prefill(prompt)["out_tokens"])
+    step = 0
+    while len(seq) < n_new:
+        done = len(seq)
+        tree = synth.plant_tree(tmpl, [-1] * tmpl.N, seq_ar[done: done + 4], seed, step, 0.6, shape.V)
+        rec = bt.step(tree)
+        seq += rec["out_tokens"]
+        step += 1
+    bt.close()
+    seq, seq_ar = seq[:n_new], seq_ar[:n_new]
+    if seq != seq_ar:
+        # a divergence is only acceptable at a position where the oracle's margin is below tolerance
+        first = next(i for i in range(n_new) if seq[i] != seq_ar[i])
+        model = oracle_model(shape, seed)
+        logits = orc.causal_logits(model, prompt + seq_ar[:first])[-1]
+        top = np.sort(logits)[::-1]
+        rms = float(np.sqrt(np.mean(logits ** 2)))
+        assert top[0] - top[1] <= LOGIT_TOL_RMS * rms, f"sequences diverge at {first} with a clear margin"
+
+
+def test_step_after_reset_reproduces_the_first_run():
+    from paper_2401_12522_b200 import Bita
+    shape = synth.CONFIGS["tiny"]
+    w = synth.make_weights(shape, 5, dtype=torch.bfloat16, device="cuda:0")
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    prompt = prompt_tokens(5, 20, shape.V)
+    b = Bita(shape, w, tmpl, C_max=256)
+    runs = []
+    for _ in range(2):
+        recs = [b.prefill(prompt)] + [b.step() for _ in range(5)]
+        runs.append([(r["out_tokens"], r["next_tree"], r["new_len"]) for r in recs])
+        b.reset()
+    assert runs[0] == runs[1]                                  # deterministic: no atomics in any reduction
+    b.close()
+
+
+def test_errors_are_reported_not_raised_by_the_device():
+    from paper_2401_12522_b200 import Bita, BitaError
+    shape = synth.CONFIGS["tiny"]
+    w = synth.make_weights(shape, 5, dtype=torch.bfloat16, device="cuda:0")
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    b = Bita(shape, w, tmpl, C_max=48)
+    with pytest.raises(BitaError) as e:
+        b.step()
+    assert e.value.code == -7                                  # not prefilled
+    with pytest.raises(BitaError) as e:
+        b.prefill(list(range(60)))
+    assert e.value.code == -3                                  # does not fit the cache
+    b.prefill(prompt_tokens(5, 20, shape.V))
+    with pytest.raises(BitaError) as e:
+        b.step([shape.V + 5] * tmpl.N)
+    assert e.value.code == -1
+    b.step()
+    with pytest.raises(BitaError) as e:
+        for _ in range(30):
+            b.step()
+    assert e.value.code == -3                                  # cache full is an error code, not a fault
+    b.close()
