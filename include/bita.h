@@ -145,12 +145,28 @@ int bita_step_finish(bita_ctx* ctx, bita_step_out* out);
 /* Back to the state after bita_init: empty cache, no last token, no tree. */
 int bita_reset(bita_ctx* ctx, bita_kv* kv);
 
+/* Cut the decoding state back (Algorithm 1 cuts the output at <EOS>; a caller that goes on after
+ * such a cut, or that explored a continuation, needs the cache cut too): keep the first `new_len`
+ * cache entries, make `last_token` the last accepted token and drop the drafted tree.
+ * 0 <= new_len <= current length. */
+int bita_rewind(bita_ctx* ctx, bita_kv* kv, int32_t new_len, int32_t last_token);
+
 /* Debugging aid for parity checks: when `dev_buf` (DEVICE, fp32) is non-NULL every
  * later pass also stores the residual stream after each layer ([L][BITA_MAX_ROWS][d],
  * the first `rows` rows of each slab valid) and the logits ([rows][V]) there, rows =
  * rows of that pass.  NULL switches it off.
  * `bytes` must hold L * BITA_MAX_ROWS * d + BITA_MAX_ROWS * V floats. */
 int bita_set_debug_buffer(bita_ctx* ctx, void* dev_buf, size_t bytes);
+
+/* Per-kernel-family device timing of later passes, for roofline reports.  When on, every
+ * projection launch and every attention launch of a pass is bracketed by CUDA events on the
+ * context's stream (a pass then runs its launches one by one instead of as one replayed graph).
+ * bita_get_kernel_timing waits for the stream and returns, for the most recent pass, the summed
+ * milliseconds and launch counts per family into HOST arrays of BITA_TIMING_FAMILIES entries:
+ * [0] projections (QKV, O, gate/up, down, LM head), [1] tree attention. */
+#define BITA_TIMING_FAMILIES 2
+int bita_set_kernel_timing(bita_ctx* ctx, int on);
+int bita_get_kernel_timing(bita_ctx* ctx, float* ms, int32_t* launches);
 
 /* Rows of the packed block of bita_step for this context (1 + N + G * n_mask). */
 int bita_block_rows(const bita_ctx* ctx);

@@ -58,7 +58,10 @@ def _signatures():
         "bita_step_enqueue": [vp, C.POINTER(KV), vp],
         "bita_step_finish": [vp, C.POINTER(StepOut)],
         "bita_reset": [vp, C.POINTER(KV)],
+        "bita_rewind": [vp, C.POINTER(KV), i32, i32],
         "bita_set_debug_buffer": [vp, vp, sz],
+        "bita_set_kernel_timing": [vp, C.c_int],
+        "bita_get_kernel_timing": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
         "bita_block_rows": [vp],
         "bita_last_launch_count": [vp],
         "bita_last_cuda_error": [],
@@ -186,6 +189,9 @@ class Bita:
     def reset(self):
         _check(lib.bita_reset(self._ctx, C.byref(self.kv)), "bita_reset")
 
+    def rewind(self, new_len: int, last_token: int):
+        _check(lib.bita_rewind(self._ctx, C.byref(self.kv), new_len, last_token), "bita_rewind")
+
     # ---- helpers ---------------------------------------------------------------------------
     def _record(self) -> Dict:
         o = self._out
@@ -210,6 +216,16 @@ class Bita:
     def debug_logits(self, rows: int) -> torch.Tensor:
         off = self.shape.L * MAX_ROWS * self.shape.d
         return self._debug[off: off + rows * self.shape.V].view(rows, self.shape.V)
+
+    def set_kernel_timing(self, on: bool):
+        _check(lib.bita_set_kernel_timing(self._ctx, 1 if on else 0), "bita_set_kernel_timing")
+
+    def kernel_timing(self):
+        """(ms, launches) per family of the most recent pass: [projections, attention]."""
+        ms = (C.c_float * 2)()
+        n = (C.c_int32 * 2)()
+        _check(lib.bita_get_kernel_timing(self._ctx, ms, n), "bita_get_kernel_timing")
+        return list(ms), list(n)
 
     @property
     def last_launch_count(self) -> int:

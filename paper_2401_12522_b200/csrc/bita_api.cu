@@ -253,11 +253,37 @@ struct bita_ctx {
   bool prefilled;
   float* dbg;
   int launches;
+  // optional per-family event timing
+  bool timing;
+  std::vector<cudaEvent_t> ev;          // pairs (start, stop)
+  std::vector<int> ev_family;           // family of each pair used by the last pass
 };
 
 namespace {
 
+// Event bracket around one launch when timing is on.
+struct Timed {
+  bita_ctx* c;
+  int slot;
+  Timed(bita_ctx* ctx, int family) : c(ctx), slot(-1) {
+    if (!c->timing) return;
+    slot = (int)c->ev_family.size();
+    if ((size_t)(2 * slot + 1) >= c->ev.size()) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { slot = -1; return; }
+      c->ev.push_back(a);
+      c->ev.push_back(b);
+    }
+    c->ev_family.push_back(family);
+    cudaEventRecord(c->ev[2 * slot], c->stream);
+  }
+  ~Timed() {
+    if (slot >= 0) cudaEventRecord(c->ev[2 * slot + 1], c->stream);
+  }
+};
+
 void gemm(bita_ctx* c, const bf16* X, const void* W, float* Y, int M, int N, int K) {
+  Timed t(c, 0);
   k_gemm_simple<<<(N + 3) / 4, 128, 0, c->stream>>>(X, (const bf16*)W, Y, M, N, K, N);
   c->launches++;
 }
@@ -280,6 +306,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   const int M = P.M;
   cudaStream_t s = c->stream;
   Buffers& b = c->b;
+  c->ev_family.clear();
   const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
   k_embed<<<M, 256, 0, s>>>(P, b.state, tree_dev, b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb,
                             m.d, m.V, b.x, b.pos, b.row_token);
@@ -297,7 +324,10 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
     a.S = attn_splits(m.H, 1); a.scale = 1.0f / sqrtf((float)m.D);
-    launch_attention(a, s);
+    {
+      Timed t(c, 1);
+      launch_attention(a, s);
+    }
     gemm(c, b.att, c->wo[l], b.tmp, M, m.d, m.H * m.D);
     k_add<<<(unsigned)(((size_t)M * m.d + 255) / 256), 256, 0, s>>>(b.x, b.tmp, (size_t)M * m.d);
     k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn);
@@ -386,6 +416,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   c->rec_host = nullptr;
   c->dbg = nullptr;
   c->launches = 0;
+  c->timing = false;
   c->prefilled = false;
   c->len_upper = 0;
   auto fail = [&](int code) { if (c->rec_host) cudaFreeHost(c->rec_host); delete c; return code; };
@@ -421,6 +452,16 @@ int bita_reset(bita_ctx* c, bita_kv* kv) {
   CU_TRY(cudaStreamSynchronize(c->stream));
   c->prefilled = false;
   c->len_upper = 0;
+  return BITA_OK;
+}
+
+int bita_rewind(bita_ctx* c, bita_kv* kv, int32_t new_len, int32_t last_token) {
+  if (!c || !kv) return BITA_ERR_INVALID_ARG;
+  if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
+  if (new_len < 0 || new_len > c->len_upper || last_token < 0 || last_token >= c->m.V) return BITA_ERR_INVALID_ARG;
+  k_set_state<<<1, 128, 0, c->stream>>>(c->b.state, new_len, last_token);
+  CU_TRY(cudaGetLastError());
+  c->len_upper = new_len;
   return BITA_OK;
 }
 
@@ -504,6 +545,26 @@ int bita_set_debug_buffer(bita_ctx* c, void* dev_buf, size_t bytes) {
   return BITA_OK;
 }
 
+int bita_set_kernel_timing(bita_ctx* c, int on) {
+  if (!c) return BITA_ERR_INVALID_ARG;
+  c->timing = on != 0;
+  c->ev_family.clear();
+  return BITA_OK;
+}
+
+int bita_get_kernel_timing(bita_ctx* c, float* ms, int32_t* launches) {
+  if (!c || !ms || !launches) return BITA_ERR_INVALID_ARG;
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  for (int f = 0; f < BITA_TIMING_FAMILIES; ++f) { ms[f] = 0.f; launches[f] = 0; }
+  for (size_t i = 0; i < c->ev_family.size(); ++i) {
+    float t = 0.f;
+    CU_TRY(cudaEventElapsedTime(&t, c->ev[2 * i], c->ev[2 * i + 1]));
+    ms[c->ev_family[i]] += t;
+    launches[c->ev_family[i]] += 1;
+  }
+  return BITA_OK;
+}
+
 int bita_block_rows(const bita_ctx* c) { return c ? c->step_plan.M : BITA_ERR_INVALID_ARG; }
 int bita_last_launch_count(const bita_ctx* c) { return c ? c->launches : BITA_ERR_INVALID_ARG; }
 
@@ -511,6 +572,7 @@ void bita_destroy(bita_ctx* c) {
   if (!c) return;
   cudaStreamSynchronize(c->stream);
   if (c->rec_host) cudaFreeHost(c->rec_host);
+  for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   delete c;
 }
 

@@ -294,6 +294,11 @@ __global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, b
   }
 }
 
+__global__ void k_set_state(DevState* st, int len, int root) {
+  if (threadIdx.x == 0) { st->len = len; st->root = root; }
+  for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
+}
+
 __global__ void k_reset_state(DevState* st) {
   if (threadIdx.x == 0) { st->len = 0; st->root = -1; st->status = 0; st->pad = 0; }
   for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
