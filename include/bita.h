@@ -38,6 +38,7 @@ extern "C" {
 #define BITA_ERR_CUDA (-5)          /* a CUDA runtime call failed; see bita_last_cuda_error           */
 #define BITA_ERR_TIMEOUT (-6)       /* a bounded device-side wait ran out (status word set)           */
 #define BITA_ERR_NOT_PREFILLED (-7) /* bita_step before bita_prefill                                  */
+#define BITA_ERR_STATIC_SCRATCH (-8) /* problem needs more than the library's built-in scratch array  */
 
 #define BITA_MAX_NODES 160          /* tree nodes, root excluded                                      */
 #define BITA_MAX_ROWS 256           /* rows of the packed block: 1 + N + G * n_mask                   */
@@ -203,6 +204,35 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
                         const int32_t* ctx_len, void* out, int32_t B, int32_t M, int32_t H,
                         int32_t H_kv, int32_t D, int32_t P, int32_t C_max, void* workspace,
                         size_t workspace_bytes, void* cuda_stream);
+
+/* Tree attention for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a serving loop whose memory pool
+ * was sized once and frozen, a plug-in that lives inside another framework's allocator, a latency
+ * path that cannot afford the device-wide synchronisation an allocation implies.  Such a caller
+ * can hold q, k, v and out, but has nowhere to get the split-KV scratch that bita_tree_attention
+ * asks for.  This variant takes the same arguments minus the workspace and keeps its scratch in a
+ * fixed array inside the library's device image: BITA_STATIC_SCRATCH_BYTES per GPU, resident on
+ * every GPU that loads the library, until the process exits.
+ *
+ * Limits and rules
+ *   - The scratch needed is what bita_attention_workspace_bytes reports for (B, M, H, D).  If that
+ *     exceeds BITA_STATIC_SCRATCH_BYTES the call returns BITA_ERR_STATIC_SCRATCH and launches
+ *     nothing.  (7B-shaped steps, H = 32, M = 69, D = 128, B = 1, fit; large batches do not.)
+ *   - The first call on each device looks up the array's device address (one runtime query, no
+ *     allocation).  Make that first call outside any stream capture.
+ *   - The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     That is harmless here, because each call overwrites every slot it later reads, but two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it: order
+ *     them on one stream or with events.
+ * Results are the same as bita_tree_attention's. */
+#define BITA_STATIC_SCRATCH_BYTES (8u << 20)
+int bita_tree_attention_static(const void* q, const void* k, const void* v, const uint32_t* vis,
+                               const void* prompt_k, const void* prompt_v, const uint8_t* sees_prompt,
+                               const int32_t* ctx_len, void* out, int32_t B, int32_t M, int32_t H,
+                               int32_t H_kv, int32_t D, int32_t P, int32_t C_max, void* cuda_stream);
 
 #ifdef __cplusplus
 }

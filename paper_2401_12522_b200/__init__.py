@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     lib,
     bita_gemm_bf16,
     bita_tree_attention,
+    bita_tree_attention_static,
     MAX_ROWS,
     MAX_NODES,
     MAX_TOPK,

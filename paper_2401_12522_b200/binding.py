@@ -69,6 +69,7 @@ def _signatures():
         "bita_gemm_bf16": [vp, vp, vp, i32, i32, i32, vp, sz, vp],
         "bita_attention_workspace_bytes": [i32, i32, i32, i32, C.POINTER(sz)],
         "bita_tree_attention": [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp],
+        "bita_tree_attention_static": [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp],
     }
 
 
@@ -272,4 +273,23 @@ def bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, 
     _check(lib.bita_tree_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(vis), _ptr(prompt_k), _ptr(prompt_v),
                                    _ptr(sees_prompt), _ptr(ctx_len), _ptr(out), B, M, H, H_kv, D, P, C_max,
                                    C.c_void_p(wp), need.value, _stream_handle(stream)), "bita_tree_attention")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def bita_tree_attention_static(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, *, H_kv, P, stream=None):
+    """Tree attention without any device allocation by the library: the caller passes inputs and
+    the output tensor, the split-KV scratch is the library's built-in array (8 MiB per GPU).
+
+    For callers that cannot allocate at call time (frozen memory pool, foreign allocator, no
+    device-wide sync allowed).  Raises BitaError(-8) when the problem needs more scratch than the
+    array holds.  Calls that overlap on the GPU share the array and race; keep them ordered.
+    """
+    B, M, H, D = q.shape
+    C_max = k.shape[2]
+    _check(lib.bita_tree_attention_static(_ptr(q), _ptr(k), _ptr(v), _ptr(vis), _ptr(prompt_k), _ptr(prompt_v),
+                                          _ptr(sees_prompt), _ptr(ctx_len), _ptr(out), B, M, H, H_kv, D, P, C_max,
+                                          _stream_handle(stream)), "bita_tree_attention_static")
     return out

@@ -586,6 +586,7 @@ const char* bita_strerror(int code) {
     case BITA_ERR_CUDA: return "CUDA runtime error";
     case BITA_ERR_TIMEOUT: return "device-side wait timed out";
     case BITA_ERR_NOT_PREFILLED: return "bita_prefill has not been called";
+    case BITA_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown error";
   }
 }
@@ -641,6 +642,50 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   launch_attention(a, (cudaStream_t)cuda_stream);
   CU_TRY(cudaGetLastError());
   return BITA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// No-allocation variant of the tree attention.  Its split-KV partials live in this fixed array of
+// the device image instead of caller-provided workspace.  Host code may not hand `g_static_scratch`
+// to a kernel (on the host the name is only a handle for the symbol): the device address is
+// looked up once per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) unsigned char g_static_scratch[BITA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+void* g_static_scratch_addr[MAX_DEVICES] = {nullptr};
+
+// Device address of the scratch array on the current device (looked up on first use).
+int static_scratch_address(void** out) {
+  int dev = -1;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return BITA_ERR_INVALID_ARG;
+  if (!g_static_scratch_addr[dev]) {
+    void* p = nullptr;
+    CU_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p || ((uintptr_t)p % ALIGN)) return BITA_ERR_CUDA;
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = g_static_scratch_addr[dev];
+  return BITA_OK;
+}
+}  // namespace
+
+int bita_tree_attention_static(const void* q, const void* k, const void* v, const uint32_t* vis, const void* prompt_k,
+                               const void* prompt_v, const uint8_t* sees_prompt, const int32_t* ctx_len, void* out,
+                               int32_t B, int32_t M, int32_t H, int32_t H_kv, int32_t D, int32_t P, int32_t C_max,
+                               void* cuda_stream) {
+  size_t need = 0;
+  int rc = bita_attention_workspace_bytes(B, M, H, D, &need);
+  if (rc) return rc;
+  if (need > BITA_STATIC_SCRATCH_BYTES) return BITA_ERR_STATIC_SCRATCH;
+  void* scratch = nullptr;
+  rc = static_scratch_address(&scratch);
+  if (rc) return rc;
+  // Every partial that the merge kernel reads is written by the slice kernel of the same call,
+  // so nothing in the shared array has to be cleared first.
+  return bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
+                             scratch, need, cuda_stream);
 }
 
 }  // extern "C"
