@@ -4,12 +4,15 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <map>
 #include <new>
+#include <tuple>
 #include <vector>
 
 #include "attention_simple.cuh"
 #include "common.cuh"
 #include "gemm_simple.cuh"
+#include "gemm_tc.cuh"
 #include "step_kernels.cuh"
 
 using namespace bita;
@@ -185,6 +188,105 @@ int check_dims(const bita_model_dims* m) {
   return BITA_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tensor-core projection: host-side planning (tensor maps, split-K, pipeline depth).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
+  return fn;
+}
+
+// bf16 matrix [rows][K] (K contiguous) -> map with a (64 x box_rows) box, 128-byte swizzle, zero fill.
+int make_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return BITA_ERR_CUDA;
+  if (((uintptr_t)base & 15) || (K % 8)) return BITA_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BLOCK_K, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return BITA_ERR_CUDA; }
+  return BITA_OK;
+}
+
+// One weight matrix (or a gate/up pair) as the projection kernel sees it.
+struct GemmDesc {
+  CUtensorMap a0, a1;
+  int N = 0, K = 0, dual = 0, tiles = 0, splits = 1, ldo = 0;
+};
+
+int gemm_splits(int tiles, int K, int max_splits) {
+  const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
+  if (tiles >= 74) return 1;
+  int s = 148 / tiles;
+  if (s > kb / 4) s = kb / 4;
+  if (s > max_splits) s = max_splits;
+  if (s < 1) s = 1;
+  return s;
+}
+
+int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
+  g->K = K;
+  g->dual = W1 ? 1 : 0;
+  int rc;
+  if (W1) {           // N = rows of each of the two matrices
+    g->tiles = (N + 63) / 64;
+    g->N = g->tiles * 128;
+    g->ldo = g->tiles * 128;
+    if ((rc = make_map(&g->a0, W0, K, N, 64))) return rc;
+    if ((rc = make_map(&g->a1, W1, K, N, 64))) return rc;
+  } else {
+    g->tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
+    g->N = N;
+    g->ldo = N;
+    if ((rc = make_map(&g->a0, W0, K, N, TC_BLOCK_N))) return rc;
+    g->a1 = g->a0;
+  }
+  g->splits = gemm_splits(g->tiles, K, max_splits);
+  return BITA_OK;
+}
+
+// Launch: X bf16 [x_rows][K] (first M rows valid) times the described weights -> out fp32 [splits][M][ldo].
+int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, float* out, int M, int32_t* status,
+                   cudaStream_t stream) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    attr_set = true;
+  }
+  GemmTcParams p{};
+  p.out = out; p.M = M; p.N = g.N; p.K = g.K; p.ldo = g.ldo; p.n_pad = n_pad; p.splits = g.splits; p.dual = g.dual;
+  p.status = status;
+  int cols = 32;
+  while (cols < n_pad) cols <<= 1;
+  p.tmem_cols = cols;
+  const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
+  const size_t budget = (n_pad <= 96 ? 110 : 220) * 1024;       // two CTAs per SM while the block is small
+  int stages = (int)((budget - 1024) / stage);
+  if (stages > 10) stages = 10;
+  if (stages < 2) stages = 2;
+  p.stages = stages;
+  const size_t smem = stages * stage + 1024;
+  dim3 grid(g.tiles, g.splits);
+  k_gemm_tc<<<grid, TC_THREADS, smem, stream>>>(g.a0, g.a1, map_b, p);
+  return BITA_OK;
+}
+
+inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
+
 int attn_splits(int H, int B) {
   int s = (148 + H * B - 1) / (H * B);
   if (s < 1) s = 1;
@@ -194,7 +296,7 @@ int attn_splits(int H, int B) {
 
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
-  float* x; bf16* xn; float* qkv; bf16* q; bf16* att; float* tmp; float* tmp2; bf16* hf; float* logits;
+  float* x; bf16* xn; float* qkv; bf16* q; bf16* att; float* tmp; float* gu; bf16* hf; float* logits;
   int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
   float2* rope_tab; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
@@ -213,11 +315,17 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   Buffers t{};
   t.x = (float*)take(R * m.d * 4);
   t.xn = (bf16*)take(R * wide * 2);
-  t.qkv = (float*)take(R * nqkv * 4);
+  // split-K partial outputs: [splits][rows][features]
+  const size_t s_qkv = gemm_splits((int)((nqkv + 127) / 128), m.d, 8);
+  const size_t s_o = gemm_splits((m.d + 127) / 128, m.H * m.D, 8);
+  const size_t s_dn = gemm_splits((m.d + 127) / 128, m.F, 8);
+  const size_t gu_tiles = (m.F + 63) / 64;
+  const size_t s_gu = gemm_splits((int)gu_tiles, m.d, 8);
+  t.qkv = (float*)take(s_qkv * R * nqkv * 4);
   t.q = (bf16*)take(R * m.H * m.D * 2);
   t.att = (bf16*)take(R * m.H * m.D * 2);
-  t.tmp = (float*)take(R * (size_t)(m.F > m.d ? m.F : m.d) * 4);
-  t.tmp2 = (float*)take(R * (size_t)m.F * 4);
+  t.tmp = (float*)take((s_o > s_dn ? s_o : s_dn) * R * (size_t)m.d * 4);
+  t.gu = (float*)take(s_gu * R * gu_tiles * 128 * 4);
   t.hf = (bf16*)take(R * (size_t)m.F * 2);
   t.logits = (float*)take(R * (size_t)m.V * 4);
   t.sel_id = (int32_t*)take(R * BITA_MAX_TOPK * 4);
@@ -253,6 +361,9 @@ struct bita_ctx {
   bool prefilled;
   float* dbg;
   int launches;
+  std::vector<GemmDesc> d_qkv, d_o, d_gu, d_dn;
+  GemmDesc d_head;
+  std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
   // optional per-family event timing
   bool timing;
   std::vector<cudaEvent_t> ev;          // pairs (start, stop)
@@ -282,10 +393,21 @@ struct Timed {
   }
 };
 
-void gemm(bita_ctx* c, const bf16* X, const void* W, float* Y, int M, int N, int K) {
+// Projection of the first M rows of an activation buffer (BITA_MAX_ROWS rows allocated).
+int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, float* out, int M) {
+  const int n_pad = pad16(M);
+  auto key = std::make_tuple((const void*)X, g.K, n_pad);
+  auto it = c->act_maps.find(key);
+  if (it == c->act_maps.end()) {
+    CUtensorMap m;
+    int rc = make_map(&m, X, g.K, BITA_MAX_ROWS, n_pad);
+    if (rc) return rc;
+    it = c->act_maps.emplace(key, m).first;
+  }
   Timed t(c, 0);
-  k_gemm_simple<<<(N + 3) / 4, 128, 0, c->stream>>>(X, (const bf16*)W, Y, M, N, K, N);
+  int rc = launch_gemm_tc(g, it->second, n_pad, out, M, &c->b.state->status, c->stream);
   c->launches++;
+  return rc;
 }
 
 void launch_attention(const AttnArgs& a, cudaStream_t s) {
@@ -312,12 +434,15 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
                             m.d, m.V, b.x, b.pos, b.row_token);
   c->launches++;
   const int nqkv = (m.H + 2 * m.H_kv) * m.D;
+  int rc;
+  k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_attn[0], m.d, m.rms_eps, b.xn);
+  c->launches++;
   for (int l = 0; l < m.L; ++l) {
     bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
     bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
-    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_attn[l], m.d, m.rms_eps, b.xn);
-    gemm(c, b.xn, c->wqkv[l], b.qkv, M, nqkv, m.d);
-    k_rope_kv<<<M, 256, 0, s>>>(b.qkv, b.pos, b.rope_tab, b.state, m.H, m.H_kv, m.D, kv->C_max, b.q, kc, vc);
+    if ((rc = gemm(c, c->d_qkv[l], b.xn, b.qkv, M))) return rc;
+    k_rope_kv<<<M, 256, 0, s>>>(b.qkv, c->d_qkv[l].splits, (size_t)M * nqkv, b.pos, b.rope_tab, b.state, m.H, m.H_kv,
+                                m.D, kv->C_max, b.q, kc, vc);
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
@@ -328,24 +453,25 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
       Timed t(c, 1);
       launch_attention(a, s);
     }
-    gemm(c, b.att, c->wo[l], b.tmp, M, m.d, m.H * m.D);
-    k_add<<<(unsigned)(((size_t)M * m.d + 255) / 256), 256, 0, s>>>(b.x, b.tmp, (size_t)M * m.d);
-    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn);
-    gemm(c, b.xn, c->wg[l], b.tmp, M, m.F, m.d);
-    gemm(c, b.xn, c->wu[l], b.tmp2, M, m.F, m.d);
-    k_swiglu<<<(unsigned)(((size_t)M * m.F + 255) / 256), 256, 0, s>>>(b.tmp, b.tmp2, (size_t)M * m.F, b.hf);
-    gemm(c, b.hf, c->wd[l], b.tmp, M, m.d, m.F);
-    k_add<<<(unsigned)(((size_t)M * m.d + 255) / 256), 256, 0, s>>>(b.x, b.tmp, (size_t)M * m.d);
-    c->launches += 8;
+    if ((rc = gemm(c, c->d_o[l], b.att, b.tmp, M))) return rc;
+    k_add_rmsnorm<<<M, 256, 0, s>>>(b.x, b.tmp, c->d_o[l].splits, (size_t)M * m.d, (const bf16*)c->g_ffn[l], m.d,
+                                    m.rms_eps, b.xn);
+    if ((rc = gemm(c, c->d_gu[l], b.xn, b.gu, M))) return rc;
+    const int ldg = c->d_gu[l].ldo;
+    k_swiglu<<<(unsigned)(((size_t)M * m.F + 255) / 256), 256, 0, s>>>(b.gu, c->d_gu[l].splits, (size_t)M * ldg, ldg,
+                                                                       m.F, M, b.hf);
+    if ((rc = gemm(c, c->d_dn[l], b.hf, b.tmp, M))) return rc;
+    const bf16* g_next = (const bf16*)(l + 1 < m.L ? c->g_attn[l + 1] : c->g_final);
+    k_add_rmsnorm<<<M, 256, 0, s>>>(b.x, b.tmp, c->d_dn[l].splits, (size_t)M * m.d, g_next, m.d, m.rms_eps, b.xn);
+    c->launches += 6;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)l * BITA_MAX_ROWS * m.d, b.x, (size_t)M * m.d * 4,
                              cudaMemcpyDeviceToDevice, s));
   }
   if (want_logits) {
-    k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_final, m.d, m.rms_eps, b.xn);
-    gemm(c, b.xn, c->lm_head, b.logits, M, m.V, m.d);
+    if ((rc = gemm(c, c->d_head, b.xn, b.logits, M))) return rc;
     k_select<<<M, 256, 0, s>>>(P, b.logits, m.V, b.sel_id, b.sel_val);
-    c->launches += 2;
+    c->launches += 1;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,
                              cudaMemcpyDeviceToDevice, s));
@@ -437,6 +563,17 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
             cudaSuccess ||
         cudaStreamSynchronize(c->stream) != cudaSuccess)
       return fail(BITA_ERR_CUDA);
+  }
+  {
+    const int nqkv = (dims->H + 2 * dims->H_kv) * dims->D;
+    c->d_qkv.resize(L); c->d_o.resize(L); c->d_gu.resize(L); c->d_dn.resize(L);
+    for (int l = 0; l < L; ++l) {
+      if ((rc = make_gemm_desc(&c->d_qkv[l], c->wqkv[l], nullptr, nqkv, dims->d, 8))) return fail(rc);
+      if ((rc = make_gemm_desc(&c->d_o[l], c->wo[l], nullptr, dims->d, dims->H * dims->D, 8))) return fail(rc);
+      if ((rc = make_gemm_desc(&c->d_gu[l], c->wg[l], c->wu[l], dims->F, dims->d, 8))) return fail(rc);
+      if ((rc = make_gemm_desc(&c->d_dn[l], c->wd[l], nullptr, dims->d, dims->F, 8))) return fail(rc);
+    }
+    if ((rc = make_gemm_desc(&c->d_head, c->lm_head, nullptr, dims->V, dims->d, 1))) return fail(rc);
   }
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
@@ -595,7 +732,8 @@ int bita_last_cuda_error(void) { return g_last_cuda_error; }
 
 int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes) {
   if (!out_bytes || M < 1 || M > BITA_MAX_ROWS || N < 1 || K < 8 || K % 8) return BITA_ERR_INVALID_ARG;
-  *out_bytes = ALIGN;
+  const int splits = gemm_splits((N + TC_BLOCK_N - 1) / TC_BLOCK_N, K, 8);
+  *out_bytes = ALIGN + align_up(splits > 1 ? (size_t)splits * M * N * 4 : 0);
   return BITA_OK;
 }
 
@@ -605,8 +743,21 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   int rc = bita_gemm_workspace_bytes(M, N, K, &need);
   if (rc) return rc;
   if (!X || !W || !Y) return BITA_ERR_INVALID_ARG;
-  if (!workspace || workspace_bytes < need) return BITA_ERR_WORKSPACE;
-  k_gemm_simple<<<(N + 3) / 4, 128, 0, (cudaStream_t)cuda_stream>>>((const bf16*)X, (const bf16*)W, (float*)Y, M, N, K, N);
+  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace % ALIGN)) return BITA_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  GemmDesc g;
+  if ((rc = make_gemm_desc(&g, W, nullptr, N, K, 8))) return rc;
+  const int n_pad = pad16(M);
+  CUtensorMap mb;
+  if ((rc = make_map(&mb, X, K, M, n_pad))) return rc;
+  int32_t* status = (int32_t*)workspace;                      // first word of the workspace: status flag
+  float* part = (float*)((uint8_t*)workspace + ALIGN);
+  CU_TRY(cudaMemsetAsync(status, 0, 4, s));
+  if ((rc = launch_gemm_tc(g, mb, n_pad, g.splits > 1 ? part : (float*)Y, M, status, s))) return rc;
+  if (g.splits > 1) {
+    const size_t n = (size_t)M * N;
+    k_reduce_splits<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, (float*)Y, n, g.splits);
+  }
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }

@@ -1,0 +1,297 @@
+// Small-M weight-streaming projection on the 5th-generation tensor cores (sm_100a).
+//
+//   Y[m][n] = sum_k X[m][k] * W[n][k]      X: bf16 [M][K] (M <= 256 rows of the packed block)
+//                                           W: bf16 [N][K] (a weight matrix, read exactly once)
+//
+// The roles are swapped with respect to a textbook GEMM: 128 weight rows are the MMA's M dimension
+// (TMEM lanes) and the block's rows, padded to a multiple of 16, are its N dimension (TMEM
+// columns).  Each CTA owns one tile of 128 output features and a contiguous range of 64-wide K
+// blocks (split-K); it streams its weight tiles through a ring of TMA-filled, 128-byte-swizzled
+// shared-memory stages, one elected thread issues tcgen05.mma into a TMEM accumulator, and four
+// epilogue warps read the accumulator back with tcgen05.ld and store fp32 results (coalesced along
+// the feature dimension).  With split-K > 1 each split stores its partial tile and the consumer
+// adds the partials in split order, which keeps every output a fixed-order sum (deterministic,
+// and independent of how many other rows the block holds).
+//
+// "Dual" mode builds the 128-row weight tile from 64 rows of each of two matrices (gate and up of
+// the SwiGLU), so that an epilogue consumer finds gate[f] and up[f] in the same tile.
+//
+// Every wait on an mbarrier is bounded: when the bound is hit the kernel raises the status word,
+// lets its copies land, frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace bita {
+
+constexpr int TC_BLOCK_N = 128;   // weight rows per tile (MMA M)
+constexpr int TC_BLOCK_K = 64;    // bf16 elements per K block = 128 bytes = one swizzle row
+constexpr int TC_UMMA_K = 16;
+constexpr int TC_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // a wait that lasts 2 s has failed
+
+struct GemmTcParams {
+  float* out;            // fp32 [splits][M][ldo] partial results (splits == 1: the result itself)
+  int32_t M;             // valid rows of X
+  int32_t N;             // output features in total (for masking the last tile); dual: 2 * F-like count per matrix
+  int32_t K;
+  int32_t ldo;           // row stride of `out` in floats
+  int32_t n_pad;         // MMA N: rows of X padded to a multiple of 16
+  int32_t stages;
+  int32_t splits;
+  int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1; output column = 2 * 64 * tile + lane-row
+  int32_t tmem_cols;     // power of two >= max(32, n_pad)
+  int32_t* status;       // device status word (sticky error flag)
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = gave up (status word raised).
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u) {
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > TC_WAIT_LIMIT_NS) break;
+    }
+  }
+  atomicExch(status, BITA_ERR_TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+// 2-D tiled TMA load global -> shared (no multicast), completion on an mbarrier.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);          // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset: next group of 8 rows
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // layout: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on an mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
+          const __grid_constant__ CUtensorMap map_b, GemmTcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[16];
+  __shared__ __align__(8) uint64_t bar_empty[16];
+  __shared__ __align__(8) uint64_t bar_acc;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int32_t abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  const int kb_total = (p.K + TC_BLOCK_K - 1) / TC_BLOCK_K;
+  const int kb0 = (int)((long)kb_total * split / p.splits);
+  const int kb1 = (int)((long)kb_total * (split + 1) / p.splits);
+  const int nkb = kb1 - kb0;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t a_bytes = TC_BLOCK_N * TC_BLOCK_K * 2;                 // 16 KiB
+  const uint32_t b_bytes = (uint32_t)p.n_pad * TC_BLOCK_K * 2;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bar_acc), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"((uint32_t)p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0 && nkb > 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      const int row_a = p.dual ? tile * 64 : tile * TC_BLOCK_N;
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+        if (i >= p.stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, p.status);
+        if (!ok) break;
+        const uint32_t full = smem_u32(&bar_full[s]);
+        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
+        const int kx = (kb0 + i) * TC_BLOCK_K;
+        mbar_expect_tx(full, stage_bytes);
+        if (p.dual) {
+          tma_load_2d(sa, &map_a0, kx, row_a, full, pol_w);
+          tma_load_2d(sa + a_bytes / 2, &map_a1, kx, row_a, full, pol_w);
+        } else {
+          tma_load_2d(sa, &map_a0, kx, row_a, full, pol_w);
+        }
+        tma_load_2d(sa + a_bytes, &map_b, kx, 0, full, pol_x);
+      }
+      if (!ok) {
+        abort_flag = 1;
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);      // let the copies in flight land
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0 && nkb > 0) {
+      const uint32_t idesc = umma_idesc(p.n_pad);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+        ok = mbar_wait(smem_u32(&bar_full[s]), ph, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
+        const uint64_t da = umma_smem_desc(sa), db = umma_smem_desc(sa + a_bytes);
+#pragma unroll
+        for (int k = 0; k < TC_BLOCK_K / TC_UMMA_K; ++k) {
+          // advancing 16 elements along K = 32 bytes = 2 units of the descriptor's address field
+          umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bar_empty[s]));                 // frees the stage when these MMAs are done
+      }
+      if (ok) umma_commit(smem_u32(&bar_acc));                // accumulator complete
+      else abort_flag = 1;
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> global (fp32)
+    const int lg = warp & 3;                                   // TMEM lane group this warp may read
+    bool ok = true;
+    if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
+    tc_fence_after();
+    if (ok) {
+      const int row_in_tile = lg * 32 + lane;
+      int n;
+      if (p.dual) n = tile * 128 + row_in_tile;                // [64 gate | 64 up] per tile, tile-major
+      else n = tile * TC_BLOCK_N + row_in_tile;
+      const bool n_ok = n < p.N;
+      float* outp = p.out + (size_t)split * p.M * p.ldo + n;
+      for (int c = 0; c < p.n_pad; c += 16) {
+        float v[16];
+        if (nkb > 0) {
+          tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+        }
+        if (n_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c + j < p.M) outp[(size_t)(c + j) * p.ldo] = v[j];
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
+                 : "memory");
+  }
+}
+
+// Y[m][n] = sum over splits, in split order.
+__global__ void k_reduce_splits(const float* __restrict__ part, float* __restrict__ y, size_t n, int splits) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float acc = part[i];
+  for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
+  y[i] = acc;
+}
+
+}  // namespace bita

@@ -61,22 +61,29 @@ __global__ void k_rmsnorm(const float* __restrict__ x, const bf16* __restrict__ 
 // Rotary embedding (half-split pairing: dims j and j + D/2) at the row's position id, then
 // q -> bf16 [M][H][D], k/v -> cache slot C + r of layout [H_kv][C_max][D].
 // rope_tab: float2 (cos, sin) [positions][D/2], computed in double on the host.
-__global__ void k_rope_kv(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
-                          const float2* __restrict__ rope_tab, const DevState* __restrict__ st, int H, int H_kv,
-                          int D, int C_max, bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc) {
+// qkv: fp32 [nsplit][M][(H + 2 H_kv) D] split-K partials, summed here in split order.
+__global__ void k_rope_kv(const float* __restrict__ qkv, int nsplit, size_t split_stride,
+                          const int32_t* __restrict__ pos, const float2* __restrict__ rope_tab,
+                          const DevState* __restrict__ st, int H, int H_kv, int D, int C_max, bf16* __restrict__ q,
+                          bf16* __restrict__ kc, bf16* __restrict__ vc) {
   const int r = blockIdx.x;
   const int half = D >> 1;
   const int p = pos[r];
   const int slot = st->len + r;
   const int nq = H * half, nk = H_kv * half;
   const float* row = qkv + (size_t)r * (H + 2 * H_kv) * D;
+  auto ld = [&](const float* ptr) {
+    float acc = ptr[0];
+    for (int sp = 1; sp < nsplit; ++sp) acc += ptr[(size_t)sp * split_stride];
+    return acc;
+  };
   for (int t = threadIdx.x; t < nq + nk; t += blockDim.x) {
     const bool isq = t < nq;
     const int u = isq ? t : t - nq;
     const int h = u / half, j = u - h * half;
     const float* src = row + (isq ? 0 : H * D) + h * D;
     const float2 cs = rope_tab[(size_t)p * half + j];
-    const float a = src[j], b = src[j + half];
+    const float a = ld(src + j), b = ld(src + j + half);
     const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
     if (isq) {
       bf16* dst = q + ((size_t)r * H + h) * D;
@@ -92,25 +99,56 @@ __global__ void k_rope_kv(const float* __restrict__ qkv, const int32_t* __restri
     const float* vsrc = row + (H + H_kv) * D;
     for (int t = threadIdx.x; t < H_kv * D; t += blockDim.x) {
       const int h = t / D, j = t - h * D;
-      vc[((size_t)h * C_max + slot) * D + j] = f2bf(vsrc[t]);
+      vc[((size_t)h * C_max + slot) * D + j] = f2bf(ld(vsrc + t));
     }
   }
 }
 
-// x += t (residual), fp32.
-__global__ void k_add(float* __restrict__ x, const float* __restrict__ t, size_t n) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) x[i] += t[i];
+// Residual add of split-K partials followed by the next RMSNorm:
+//   x[r] += sum_s part[s][r]   (split order);   xn[r] = x[r] * g / sqrt(mean(x[r]^2) + eps)  (bf16)
+// One block per row.
+__global__ void k_add_rmsnorm(float* __restrict__ x, const float* __restrict__ part, int nsplit, size_t split_stride,
+                              const bf16* __restrict__ g, int d, float eps, bf16* __restrict__ xn) {
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  float* xr = x + (size_t)r * d;
+  const float* pr = part + (size_t)r * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = xr[c];
+    for (int sp = 0; sp < nsplit; ++sp) v += pr[(size_t)sp * split_stride + c];
+    xr[c] = v;
+    ss += v * v;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
+  }
+  __syncthreads();
+  const float inv = red[0];
+  bf16* o = xn + (size_t)r * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
 }
 
-// hf = silu(gate) * up -> bf16.  gate/up fp32 [M][F].
-__global__ void k_swiglu(const float* __restrict__ gate, const float* __restrict__ up, size_t n,
+// hf[r][f] = silu(gate) * up -> bf16, from the dual-tile projection output: fp32
+// [nsplit][M][ldg] where tile t holds gate features 64t..64t+63 in columns 128t..128t+63 and the
+// matching up features in columns 128t+64..128t+127.
+__global__ void k_swiglu(const float* __restrict__ gu, int nsplit, size_t split_stride, int ldg, int F, int M,
                          bf16* __restrict__ hf) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) {
-    const float g = gate[i];
-    hf[i] = f2bf(g / (1.0f + __expf(-g)) * up[i]);
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)M * F) return;
+  const int r = (int)(i / F), f = (int)(i - (size_t)r * F);
+  const float* src = gu + (size_t)r * ldg + (f >> 6) * 128 + (f & 63);
+  float g = 0.f, u = 0.f;
+  for (int sp = 0; sp < nsplit; ++sp) {
+    g += src[(size_t)sp * split_stride];
+    u += src[(size_t)sp * split_stride + 64];
   }
+  hf[i] = f2bf(g / (1.0f + __expf(-g)) * u);
 }
 
 // ---------------------------------------------------------------------------------------------
