@@ -264,7 +264,7 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, float
                    cudaStream_t stream) {
   static bool attr_set = false;
   if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     attr_set = true;
   }
   GemmTcParams p{};
