@@ -9,7 +9,7 @@
 #include <tuple>
 #include <vector>
 
-#include "attention_simple.cuh"
+#include "attention_tc.cuh"
 #include "common.cuh"
 #include "gemm_simple.cuh"
 #include "gemm_tc.cuh"
@@ -287,10 +287,21 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, float
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
 
-int attn_splits(int H, int B) {
-  int s = (148 + H * B - 1) / (H * B);
+// Attention launch shape: warps per CTA, row tiles, key slices (about two CTAs per SM in total).
+void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
+  int w = (M + 15) / 16;
+  if (w > 8) w = 8;
+  const int rt = (M + 16 * w - 1) / (16 * w);
+  const int ctas = H * B * rt;
+  int s = (296 + ctas - 1) / ctas;
   if (s < 1) s = 1;
-  if (s > 8) s = 8;
+  if (s > 6) s = 6;
+  *warps = w; *row_tiles = rt; *splits = s;
+}
+
+int attn_splits(int H, int B, int M) {
+  int w, rt, s;
+  attn_shape(H, B, M, &w, &rt, &s);
   return s;
 }
 
@@ -332,7 +343,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.sel_val = (float*)take(R * BITA_MAX_TOPK * 4);
   t.pos = (int32_t*)take(R * 4);
   t.row_token = (int32_t*)take(R * 4);
-  const size_t S = attn_splits(m.H, 1);
+  const size_t S = 6;                        // upper bound of attn_splits
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
@@ -410,15 +421,28 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, float* out, int M) {
   return rc;
 }
 
-void launch_attention(const AttnArgs& a, cudaStream_t s) {
-  dim3 g1(a.H, a.S, a.B), g2(a.M, a.H, a.B);
-  if (a.D == 128) {
-    k_attn_simple<128><<<g1, 128, 0, s>>>(a);
-    k_attn_merge<128><<<g2, 128, 0, s>>>(a);
-  } else {
-    k_attn_simple<64><<<g1, 128, 0, s>>>(a);
-    k_attn_merge<64><<<g2, 64, 0, s>>>(a);
+// Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches slices + merge.
+int launch_attention(AttnArgs a, cudaStream_t s) {
+  attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
+  const int rows_cta = a.warps * 16;
+  const size_t smem = (size_t)rows_cta * a.D * 2 + 4 * (size_t)ATT_KEYS * a.D * 2 + (size_t)rows_cta * a.W * 4 +
+                      rows_cta + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    attr_set = true;
   }
+  dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
+  if (a.D == 128) {
+    k_attn_tc<128><<<g1, a.warps * 32, smem, s>>>(a);
+    k_attn_merge<128><<<g2, 64, 0, s>>>(a);
+  } else {
+    k_attn_tc<64><<<g1, a.warps * 32, smem, s>>>(a);
+    k_attn_merge<64><<<g2, 32, 0, s>>>(a);
+  }
+  return BITA_OK;
 }
 
 // The layer stack over one packed block, then (optionally) the LM head and selection.
@@ -448,10 +472,9 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
-    a.S = attn_splits(m.H, 1); a.scale = 1.0f / sqrtf((float)m.D);
     {
       Timed t(c, 1);
-      launch_attention(a, s);
+      if ((rc = launch_attention(a, s))) return rc;
     }
     if ((rc = gemm(c, c->d_o[l], b.att, b.tmp, M))) return rc;
     k_add_rmsnorm<<<M, 256, 0, s>>>(b.x, b.tmp, c->d_o[l].splits, (size_t)M * m.d, (const bf16*)c->g_ffn[l], m.d,
@@ -764,7 +787,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
 
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
   if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
-  const size_t S = attn_splits(H, B);
+  const size_t S = attn_splits(H, B, M);
   *out_bytes = align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
   return BITA_OK;
 }
@@ -785,12 +808,10 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
   a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
-  a.S = attn_splits(H, B);
   a.part_ml = (float*)workspace;
-  a.part_acc = (float*)((uint8_t*)workspace + align_up((size_t)B * H * a.S * M * 2 * 4));
+  a.part_acc = (float*)((uint8_t*)workspace + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  a.scale = 1.0f / sqrtf((float)D);
-  launch_attention(a, (cudaStream_t)cuda_stream);
+  if ((rc = launch_attention(a, (cudaStream_t)cuda_stream))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }
