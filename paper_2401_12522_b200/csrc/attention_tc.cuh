@@ -82,6 +82,8 @@ __global__ void __launch_bounds__(256) k_attn_tc(AttnArgs a) {
   constexpr int KS_Q = D / 16;               // k-steps of Q.K^T
   constexpr int KS_P = ATT_KEYS / 16;        // k-steps of P.V
   extern __shared__ __align__(128) uint8_t smem[];
+  pdl_launch();
+  pdl_wait();
   const int h = blockIdx.x, s = blockIdx.y;
   const int b = blockIdx.z / a.row_tiles, rt = blockIdx.z - b * a.row_tiles;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -290,6 +292,8 @@ __global__ void __launch_bounds__(256) k_attn_tc(AttnArgs a) {
 // grid = (M, H, B), D / 2 threads (one float2 of the output each).
 template <int D>
 __global__ void k_attn_merge(AttnArgs a) {
+  pdl_launch();
+  pdl_wait();
   const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const size_t p0 = (((size_t)b * a.H + h) * a.S) * a.M + r;
   float mx = -INFINITY;

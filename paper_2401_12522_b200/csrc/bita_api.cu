@@ -2,6 +2,7 @@
 // launch sequence of one pass.  Every step of the pass runs in the kernels included below.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -11,7 +12,6 @@
 
 #include "attention_tc.cuh"
 #include "common.cuh"
-#include "gemm_simple.cuh"
 #include "gemm_tc.cuh"
 #include "step_kernels.cuh"
 
@@ -29,6 +29,35 @@ thread_local int g_last_cuda_error = 0;
       return BITA_ERR_CUDA;                            \
     }                                                  \
   } while (0)
+
+// Launch with optional thread-block cluster along y and optional programmatic dependent launch.
+template <typename... P, typename... A>
+int launch(cudaStream_t s, bool pdl, dim3 grid, dim3 block, size_t smem, unsigned cluster_y, void (*kernel)(P...),
+           A... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  unsigned n = 0;
+  if (cluster_y > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = 1;
+    at[n].val.clusterDim.y = cluster_y;
+    at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n;
+  CU_TRY(cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...));
+  return BITA_OK;
+}
 
 constexpr int PREFILL_CHUNK = 128;
 constexpr size_t ALIGN = 256;
@@ -225,15 +254,16 @@ int make_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows) {
 // One weight matrix (or a gate/up pair) as the projection kernel sees it.
 struct GemmDesc {
   CUtensorMap a0, a1;
-  int N = 0, K = 0, dual = 0, tiles = 0, splits = 1, ldo = 0;
+  int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
 };
 
+// Split-K factor (= cluster size): enough CTAs for about two per SM, at least 4 K blocks each.
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  if (tiles >= 74) return 1;
-  int s = 148 / tiles;
+  int s = (296 + tiles / 2) / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
+  if (s > 8) s = 8;
   if (s < 1) s = 1;
   return s;
 }
@@ -244,14 +274,12 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
   int rc;
   if (W1) {           // N = rows of each of the two matrices
     g->tiles = (N + 63) / 64;
-    g->N = g->tiles * 128;
-    g->ldo = g->tiles * 128;
+    g->N = N;
     if ((rc = make_map(&g->a0, W0, K, N, 64))) return rc;
     if ((rc = make_map(&g->a1, W1, K, N, 64))) return rc;
   } else {
     g->tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
     g->N = N;
-    g->ldo = N;
     if ((rc = make_map(&g->a0, W0, K, N, TC_BLOCK_N))) return rc;
     g->a1 = g->a0;
   }
@@ -259,17 +287,15 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
   return BITA_OK;
 }
 
-// Launch: X bf16 [x_rows][K] (first M rows valid) times the described weights -> out fp32 [splits][M][ldo].
-int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, float* out, int M, int32_t* status,
+// Launch: X bf16 (first M rows valid) times the described weights; `p` carries the epilogue.
+int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M, GemmTcParams p, bool pdl,
                    cudaStream_t stream) {
   static bool attr_set = false;
   if (!attr_set) {
     CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     attr_set = true;
   }
-  GemmTcParams p{};
-  p.out = out; p.M = M; p.N = g.N; p.K = g.K; p.ldo = g.ldo; p.n_pad = n_pad; p.splits = g.splits; p.dual = g.dual;
-  p.status = status;
+  p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.splits = g.splits; p.dual = g.dual;
   int cols = 32;
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
@@ -278,11 +304,11 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, float
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
+  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // reduction buffer
   p.stages = stages;
   const size_t smem = stages * stage + 1024;
-  dim3 grid(g.tiles, g.splits);
-  k_gemm_tc<<<grid, TC_THREADS, smem, stream>>>(g.a0, g.a1, map_b, p);
-  return BITA_OK;
+  return launch(stream, pdl, dim3(g.tiles, g.splits), dim3(TC_THREADS), smem, (unsigned)g.splits, k_gemm_tc, g.a0,
+                g.a1, map_b, p);
 }
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
@@ -307,7 +333,7 @@ int attn_splits(int H, int B, int M) {
 
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
-  float* x; bf16* xn; float* qkv; bf16* q; bf16* att; float* tmp; float* gu; bf16* hf; float* logits;
+  float* x; bf16* xn; bf16* q; bf16* att; float* tmp; bf16* hf; float* logits;
   int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
   float2* rope_tab; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
@@ -321,22 +347,13 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
     return p;
   };
   const size_t R = BITA_MAX_ROWS;
-  const size_t nqkv = (size_t)(m.H + 2 * m.H_kv) * m.D;
   const size_t wide = (size_t)m.d > (size_t)m.H * m.D ? m.d : (size_t)m.H * m.D;
   Buffers t{};
   t.x = (float*)take(R * m.d * 4);
   t.xn = (bf16*)take(R * wide * 2);
-  // split-K partial outputs: [splits][rows][features]
-  const size_t s_qkv = gemm_splits((int)((nqkv + 127) / 128), m.d, 8);
-  const size_t s_o = gemm_splits((m.d + 127) / 128, m.H * m.D, 8);
-  const size_t s_dn = gemm_splits((m.d + 127) / 128, m.F, 8);
-  const size_t gu_tiles = (m.F + 63) / 64;
-  const size_t s_gu = gemm_splits((int)gu_tiles, m.d, 8);
-  t.qkv = (float*)take(s_qkv * R * nqkv * 4);
   t.q = (bf16*)take(R * m.H * m.D * 2);
   t.att = (bf16*)take(R * m.H * m.D * 2);
-  t.tmp = (float*)take((s_o > s_dn ? s_o : s_dn) * R * (size_t)m.d * 4);
-  t.gu = (float*)take(s_gu * R * gu_tiles * 128 * 4);
+  t.tmp = (float*)take(R * (size_t)m.d * 4);
   t.hf = (bf16*)take(R * (size_t)m.F * 2);
   t.logits = (float*)take(R * (size_t)m.V * 4);
   t.sel_id = (int32_t*)take(R * BITA_MAX_TOPK * 4);
@@ -375,6 +392,7 @@ struct bita_ctx {
   std::vector<GemmDesc> d_qkv, d_o, d_gu, d_dn;
   GemmDesc d_head;
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
+  bool pdl;                             // programmatic dependent launch between the kernels of a pass
   // optional per-family event timing
   bool timing;
   std::vector<cudaEvent_t> ev;          // pairs (start, stop)
@@ -405,7 +423,7 @@ struct Timed {
 };
 
 // Projection of the first M rows of an activation buffer (BITA_MAX_ROWS rows allocated).
-int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, float* out, int M) {
+int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   const int n_pad = pad16(M);
   auto key = std::make_tuple((const void*)X, g.K, n_pad);
   auto it = c->act_maps.find(key);
@@ -415,14 +433,21 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, float* out, int M) {
     if (rc) return rc;
     it = c->act_maps.emplace(key, m).first;
   }
+  p.status = &c->b.state->status;
   Timed t(c, 0);
-  int rc = launch_gemm_tc(g, it->second, n_pad, out, M, &c->b.state->status, c->stream);
+  int rc = launch_gemm_tc(g, it->second, n_pad, M, p, c->pdl, c->stream);
   c->launches++;
   return rc;
 }
 
+GemmTcParams epi_store(float* out, int ldo) {
+  GemmTcParams p{};
+  p.mode = EPI_STORE; p.out = out; p.ldo = ldo;
+  return p;
+}
+
 // Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches slices + merge.
-int launch_attention(AttnArgs a, cudaStream_t s) {
+int launch_attention(AttnArgs a, bool pdl, cudaStream_t s) {
   attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const int rows_cta = a.warps * 16;
@@ -435,14 +460,13 @@ int launch_attention(AttnArgs a, cudaStream_t s) {
     attr_set = true;
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
+  int rc;
   if (a.D == 128) {
-    k_attn_tc<128><<<g1, a.warps * 32, smem, s>>>(a);
-    k_attn_merge<128><<<g2, 64, 0, s>>>(a);
-  } else {
-    k_attn_tc<64><<<g1, a.warps * 32, smem, s>>>(a);
-    k_attn_merge<64><<<g2, 32, 0, s>>>(a);
+    if ((rc = launch(s, pdl, g1, dim3(a.warps * 32), smem, 1, k_attn_tc<128>, a))) return rc;
+    return launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a);
   }
-  return BITA_OK;
+  if ((rc = launch(s, pdl, g1, dim3(a.warps * 32), smem, 1, k_attn_tc<64>, a))) return rc;
+  return launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
 
 // The layer stack over one packed block, then (optionally) the LM head and selection.
@@ -454,19 +478,25 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   Buffers& b = c->b;
   c->ev_family.clear();
   const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
-  k_embed<<<M, 256, 0, s>>>(P, b.state, tree_dev, b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb,
-                            m.d, m.V, b.x, b.pos, b.row_token);
-  c->launches++;
-  const int nqkv = (m.H + 2 * m.H_kv) * m.D;
+  const bool pdl = c->pdl;
   int rc;
-  k_rmsnorm<<<M, 256, 0, s>>>(b.x, (const bf16*)c->g_attn[0], m.d, m.rms_eps, b.xn);
-  c->launches++;
+  if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_embed, P, (const DevState*)b.state, tree_dev,
+                   (const int32_t*)b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb, m.d, m.V, b.x,
+                   b.pos, b.row_token)))
+    return rc;
+  if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_rmsnorm, (const float*)b.x, (const bf16*)c->g_attn[0], m.d,
+                   m.rms_eps, b.xn)))
+    return rc;
+  c->launches += 2;
   for (int l = 0; l < m.L; ++l) {
     bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
     bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
-    if ((rc = gemm(c, c->d_qkv[l], b.xn, b.qkv, M))) return rc;
-    k_rope_kv<<<M, 256, 0, s>>>(b.qkv, c->d_qkv[l].splits, (size_t)M * nqkv, b.pos, b.rope_tab, b.state, m.H, m.H_kv,
-                                m.D, kv->C_max, b.q, kc, vc);
+    {   // q, k, v projection + rotary embedding + cache write
+      GemmTcParams p{};
+      p.mode = EPI_QKV; p.q = b.q; p.kc = kc; p.vc = vc; p.pos = b.pos; p.rope_tab = b.rope_tab;
+      p.len_ptr = &b.state->len; p.H = m.H; p.H_kv = m.H_kv; p.D = m.D; p.C_max = kv->C_max;
+      if ((rc = gemm(c, c->d_qkv[l], b.xn, M, p))) return rc;
+    }
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
@@ -474,26 +504,31 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
     {
       Timed t(c, 1);
-      if ((rc = launch_attention(a, s))) return rc;
+      if ((rc = launch_attention(a, pdl, s))) return rc;
     }
-    if ((rc = gemm(c, c->d_o[l], b.att, b.tmp, M))) return rc;
-    k_add_rmsnorm<<<M, 256, 0, s>>>(b.x, b.tmp, c->d_o[l].splits, (size_t)M * m.d, (const bf16*)c->g_ffn[l], m.d,
-                                    m.rms_eps, b.xn);
-    if ((rc = gemm(c, c->d_gu[l], b.xn, b.gu, M))) return rc;
-    const int ldg = c->d_gu[l].ldo;
-    k_swiglu<<<(unsigned)(((size_t)M * m.F + 255) / 256), 256, 0, s>>>(b.gu, c->d_gu[l].splits, (size_t)M * ldg, ldg,
-                                                                       m.F, M, b.hf);
-    if ((rc = gemm(c, c->d_dn[l], b.hf, b.tmp, M))) return rc;
+    if ((rc = gemm(c, c->d_o[l], b.att, M, epi_store(b.tmp, m.d)))) return rc;
+    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp,
+                     (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn)))
+      return rc;
+    {   // gate/up projection + SwiGLU
+      GemmTcParams p{};
+      p.mode = EPI_SWIGLU; p.hf = b.hf; p.F = m.F;
+      if ((rc = gemm(c, c->d_gu[l], b.xn, M, p))) return rc;
+    }
+    if ((rc = gemm(c, c->d_dn[l], b.hf, M, epi_store(b.tmp, m.d)))) return rc;
     const bf16* g_next = (const bf16*)(l + 1 < m.L ? c->g_attn[l + 1] : c->g_final);
-    k_add_rmsnorm<<<M, 256, 0, s>>>(b.x, b.tmp, c->d_dn[l].splits, (size_t)M * m.d, g_next, m.d, m.rms_eps, b.xn);
-    c->launches += 6;
+    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp, g_next, m.d,
+                     m.rms_eps, b.xn)))
+      return rc;
+    c->launches += 4;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)l * BITA_MAX_ROWS * m.d, b.x, (size_t)M * m.d * 4,
                              cudaMemcpyDeviceToDevice, s));
   }
   if (want_logits) {
-    if ((rc = gemm(c, c->d_head, b.xn, b.logits, M))) return rc;
-    k_select<<<M, 256, 0, s>>>(P, b.logits, m.V, b.sel_id, b.sel_val);
+    if ((rc = gemm(c, c->d_head, b.xn, M, epi_store(b.logits, m.V)))) return rc;
+    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select, P, (const float*)b.logits, m.V, b.sel_id, b.sel_val)))
+      return rc;
     c->launches += 1;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,
@@ -566,6 +601,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   c->dbg = nullptr;
   c->launches = 0;
   c->timing = false;
+  c->pdl = getenv("BITA_NO_PDL") == nullptr;
   c->prefilled = false;
   c->len_upper = 0;
   auto fail = [&](int code) { if (c->rec_host) cudaFreeHost(c->rec_host); delete c; return code; };
@@ -641,8 +677,9 @@ int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count,
     CU_TRY(cudaMemcpyAsync(c->b.query_tokens, tokens + done, cnt * 4, cudaMemcpyHostToDevice, c->stream));
     rc = run_block(c, kv, c->prefill_plan, nullptr, last);
     if (rc) return rc;
-    k_prefill_finish<<<1, 32, 0, c->stream>>>(c->prefill_plan.dev, c->step_plan.dev, c->b.state, c->b.sel_id, c->b.rec,
-                                              last ? 1 : 0);
+    if ((rc = launch(c->stream, c->pdl, dim3(1), dim3(32), 0, 1, k_prefill_finish, c->prefill_plan.dev,
+                     c->step_plan.dev, c->b.state, (const int32_t*)c->b.sel_id, c->b.rec, last ? 1 : 0)))
+      return rc;
     c->launches++;
     CU_TRY(cudaStreamSynchronize(c->stream));   // the plan region and token buffer are reused by the next chunk
     done += cnt;
@@ -663,8 +700,12 @@ int bita_step_enqueue(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens_dev) 
   c->launches = 0;
   int rc = run_block(c, kv, c->step_plan, tree_tokens_dev, true);
   if (rc) return rc;
-  k_accept<<<1, 32, 0, c->stream>>>(c->step_plan.dev, c->b.state, c->b.row_token, c->b.sel_id, c->b.rec);
-  k_compact<<<c->m.L * c->m.H_kv, 64, 0, c->stream>>>(c->b.rec, c->m.D, kv->C_max, (bf16*)kv->k, (bf16*)kv->v);
+  if ((rc = launch(c->stream, c->pdl, dim3(1), dim3(32), 0, 1, k_accept, c->step_plan.dev, c->b.state,
+                   (const int32_t*)c->b.row_token, (const int32_t*)c->b.sel_id, c->b.rec)))
+    return rc;
+  if ((rc = launch(c->stream, c->pdl, dim3(c->m.L * c->m.H_kv), dim3(64), 0, 1, k_compact, (const DevRecord*)c->b.rec,
+                   c->m.D, kv->C_max, (bf16*)kv->k, (bf16*)kv->v)))
+    return rc;
   c->launches += 2;
   CU_TRY(cudaGetLastError());
   CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
@@ -755,8 +796,7 @@ int bita_last_cuda_error(void) { return g_last_cuda_error; }
 
 int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes) {
   if (!out_bytes || M < 1 || M > BITA_MAX_ROWS || N < 1 || K < 8 || K % 8) return BITA_ERR_INVALID_ARG;
-  const int splits = gemm_splits((N + TC_BLOCK_N - 1) / TC_BLOCK_N, K, 8);
-  *out_bytes = ALIGN + align_up(splits > 1 ? (size_t)splits * M * N * 4 : 0);
+  *out_bytes = ALIGN;                                         // one status word
   return BITA_OK;
 }
 
@@ -773,14 +813,10 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   const int n_pad = pad16(M);
   CUtensorMap mb;
   if ((rc = make_map(&mb, X, K, M, n_pad))) return rc;
-  int32_t* status = (int32_t*)workspace;                      // first word of the workspace: status flag
-  float* part = (float*)((uint8_t*)workspace + ALIGN);
-  CU_TRY(cudaMemsetAsync(status, 0, 4, s));
-  if ((rc = launch_gemm_tc(g, mb, n_pad, g.splits > 1 ? part : (float*)Y, M, status, s))) return rc;
-  if (g.splits > 1) {
-    const size_t n = (size_t)M * N;
-    k_reduce_splits<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, (float*)Y, n, g.splits);
-  }
+  CU_TRY(cudaMemsetAsync(workspace, 0, 4, s));
+  GemmTcParams p = epi_store((float*)Y, N);
+  p.status = (int32_t*)workspace;
+  if ((rc = launch_gemm_tc(g, mb, n_pad, M, p, false, s))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }
@@ -811,7 +847,7 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   a.part_ml = (float*)workspace;
   a.part_acc = (float*)((uint8_t*)workspace + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  if ((rc = launch_attention(a, (cudaStream_t)cuda_stream))) return rc;
+  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }

@@ -65,6 +65,12 @@ __device__ __forceinline__ bf16 f2bf(float v) { return __float2bfloat16_rn(v); }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// Programmatic dependent launch: `pdl_launch` lets the next kernel of the stream begin its own
+// prologue; `pdl_wait` blocks until every kernel this one depends on has completed and its writes
+// are visible.  A kernel must not touch memory that earlier kernels write before `pdl_wait`.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -8,13 +8,18 @@
 // columns).  Each CTA owns one tile of 128 output features and a contiguous range of 64-wide K
 // blocks (split-K); it streams its weight tiles through a ring of TMA-filled, 128-byte-swizzled
 // shared-memory stages, one elected thread issues tcgen05.mma into a TMEM accumulator, and four
-// epilogue warps read the accumulator back with tcgen05.ld and store fp32 results (coalesced along
-// the feature dimension).  With split-K > 1 each split stores its partial tile and the consumer
-// adds the partials in split order, which keeps every output a fixed-order sum (deterministic,
-// and independent of how many other rows the block holds).
+// epilogue warps read the accumulator back with tcgen05.ld.  The splits of one tile form a
+// thread-block cluster: every split parks its partial tile in its own shared memory, and after a
+// cluster barrier each split sums a slice of the rows over all partners through distributed shared
+// memory, always in split order - every output is a fixed-order sum (deterministic, and
+// independent of how many other rows the block holds) and no partial result ever goes to HBM.
+// The reducing thread then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
+// builds the 128-row weight tile from 64 gate rows and the 64 matching up rows, so both halves of
+// a product sit in the same tile); or rotary embedding with the q rows going to a bf16 buffer and
+// the k/v rows straight into the KV cache.
 //
-// "Dual" mode builds the 128-row weight tile from 64 rows of each of two matrices (gate and up of
-// the SwiGLU), so that an epilogue consumer finds gate[f] and up[f] in the same tile.
+// Programmatic dependent launch: the weight tiles of the first ring fill are requested before
+// the kernel waits for its predecessor, so HBM stays busy across the kernel boundary.
 //
 // Every wait on an mbarrier is bounded: when the bound is hit the kernel raises the status word,
 // lets its copies land, frees its TMEM and returns.
@@ -32,18 +37,37 @@ constexpr int TC_UMMA_K = 16;
 constexpr int TC_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // a wait that lasts 2 s has failed
 
+enum GemmEpilogue : int32_t {
+  EPI_STORE = 0,    // out[m][n] = y                                   (fp32)
+  EPI_SWIGLU = 1,   // dual tile: hf[m][f] = silu(gate) * up            (bf16)
+  EPI_QKV = 2,      // rotary embedding, q -> bf16 buffer, k/v -> cache (bf16)
+};
+
 struct GemmTcParams {
-  float* out;            // fp32 [splits][M][ldo] partial results (splits == 1: the result itself)
   int32_t M;             // valid rows of X
-  int32_t N;             // output features in total (for masking the last tile); dual: 2 * F-like count per matrix
+  int32_t N;             // output features (for masking the last tile)
   int32_t K;
-  int32_t ldo;           // row stride of `out` in floats
   int32_t n_pad;         // MMA N: rows of X padded to a multiple of 16
   int32_t stages;
-  int32_t splits;
-  int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1; output column = 2 * 64 * tile + lane-row
+  int32_t splits;        // = cluster size along y; split s of a tile is cluster rank s
+  int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1
   int32_t tmem_cols;     // power of two >= max(32, n_pad)
+  int32_t mode;          // GemmEpilogue
   int32_t* status;       // device status word (sticky error flag)
+  // EPI_STORE
+  float* out;            // fp32 [M][ldo]
+  int32_t ldo;
+  // EPI_SWIGLU
+  bf16* hf;              // bf16 [M][F]
+  int32_t F;
+  // EPI_QKV
+  bf16* q;               // bf16 [M][H][D]
+  bf16* kc;              // this layer's key cache   [H_kv][C_max][D]
+  bf16* vc;              // this layer's value cache
+  const int32_t* pos;    // position id of each row
+  const float2* rope_tab;  // (cos, sin) [position][D/2]
+  const int32_t* len_ptr;  // cache length C (device)
+  int32_t H, H_kv, D, C_max;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -151,6 +175,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Thread-block cluster helpers (split-K partners form one cluster).
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float dsmem_ld(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
@@ -160,7 +206,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t bar_empty[16];
   __shared__ __align__(8) uint64_t bar_acc;
   __shared__ uint32_t tmem_base_slot;
-  __shared__ int32_t abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -180,7 +225,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     mbar_init(smem_u32(&bar_acc), 1);
-    abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -194,17 +238,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
+  if (threadIdx.x == 0) pdl_launch();          // the next kernel may start its prologue
+
   if (warp == 0) {
     // ---------------- TMA producer
     if (lane == 0 && nkb > 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       const int row_a = p.dual ? tile * 64 : tile * TC_BLOCK_N;
-      bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
+      auto load_a = [&](int i) {
         const int s = i % p.stages;
-        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        if (i >= p.stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, p.status);
-        if (!ok) break;
         const uint32_t full = smem_u32(&bar_full[s]);
         const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
         const int kx = (kb0 + i) * TC_BLOCK_K;
@@ -215,10 +257,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         } else {
           tma_load_2d(sa, &map_a0, kx, row_a, full, pol_w);
         }
-        tma_load_2d(sa + a_bytes, &map_b, kx, 0, full, pol_x);
+      };
+      auto load_b = [&](int i) {
+        const int s = i % p.stages;
+        tma_load_2d(smem_base + (uint32_t)s * stage_bytes + a_bytes, &map_b, (kb0 + i) * TC_BLOCK_K, 0,
+                    smem_u32(&bar_full[s]), pol_x);
+      };
+      // weights do not depend on earlier kernels: fill the ring with them first, then wait for
+      // the producer of the activations
+      const int npre = nkb < p.stages ? nkb : p.stages;
+      for (int i = 0; i < npre; ++i) load_a(i);
+      pdl_wait();
+      for (int i = 0; i < npre; ++i) load_b(i);
+      bool ok = true;
+      for (int i = npre; i < nkb; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+        ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, p.status);
+        if (!ok) break;
+        load_a(i);
+        load_b(i);
       }
       if (!ok) {
-        abort_flag = 1;
         for (int i = 0; i < 64; ++i) __nanosleep(1000);      // let the copies in flight land
       }
     }
@@ -243,53 +303,134 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         umma_commit(smem_u32(&bar_empty[s]));                 // frees the stage when these MMAs are done
       }
       if (ok) umma_commit(smem_u32(&bar_acc));                // accumulator complete
-      else abort_flag = 1;
     }
-  } else {
-    // ---------------- epilogue: TMEM -> registers -> global (fp32)
-    const int lg = warp & 3;                                   // TMEM lane group this warp may read
+  }
+
+  // ---------------- epilogue, part 1: this split's partial tile TMEM -> shared memory
+  // red[token][feature] (fp32) reuses the pipeline stages: every copy has landed and every MMA has
+  // read its operands once the accumulator barrier has completed.
+  float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+  const int lg = warp & 3;                                     // TMEM lane group this warp may read
+  const int fr = lg * 32 + lane;                               // feature row of the tile owned by this thread
+  if (warp >= 2) {
     bool ok = true;
     if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     tc_fence_after();
-    if (ok) {
-      const int row_in_tile = lg * 32 + lane;
-      int n;
-      if (p.dual) n = tile * 128 + row_in_tile;                // [64 gate | 64 up] per tile, tile-major
-      else n = tile * TC_BLOCK_N + row_in_tile;
-      const bool n_ok = n < p.N;
-      float* outp = p.out + (size_t)split * p.M * p.ldo + n;
-      for (int c = 0; c < p.n_pad; c += 16) {
-        float v[16];
-        if (nkb > 0) {
-          tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, v);
-        } else {
+    for (int c = 0; c < p.n_pad; c += 16) {
+      float v[16];
+      if (nkb > 0 && ok) {
+        tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, v);
+      } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+        for (int j = 0; j < 16; ++j) v[j] = 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (c + j < p.M) red[(c + j) * TC_BLOCK_N + fr] = v[j];
+    }
+  }
+  tc_fence_before();
+  __syncwarp();
+  cluster_sync_all();                                          // partial tiles of all splits are in place
+
+  // ---------------- epilogue, part 2: each split reduces a slice of the rows over all splits, in
+  // split order, and applies the fused operation.  Rows are handled eight at a time so that the
+  // (remote) shared-memory and global loads of a batch are in flight together.
+  if (warp >= 2) {
+    constexpr int TB = 8;
+    pdl_wait();
+    const int rank = (int)cluster_rank();
+    const int per = (p.M + p.splits - 1) / p.splits;
+    const int t0 = rank * per, t1 = min(p.M, t0 + per);
+    const uint32_t red_u32 = smem_base;
+    const int n = tile * TC_BLOCK_N + fr;                      // output feature (EPI_STORE / EPI_QKV)
+    for (int tok0 = t0; tok0 < t1; tok0 += TB) {
+      float acc[TB];
+#pragma unroll
+      for (int u = 0; u < TB; ++u) acc[u] = 0.f;
+      if (p.splits == 1) {
+#pragma unroll
+        for (int u = 0; u < TB; ++u)
+          if (tok0 + u < t1) acc[u] = red[(tok0 + u) * TC_BLOCK_N + fr];
+      } else {
+        for (int r = 0; r < p.splits; ++r) {
+          const uint32_t base = dsmem_addr(red_u32, (uint32_t)r) + (uint32_t)fr * 4u;
+          float v[TB];
+#pragma unroll
+          for (int u = 0; u < TB; ++u)
+            v[u] = (tok0 + u < t1) ? dsmem_ld(base + (uint32_t)((tok0 + u) * TC_BLOCK_N) * 4u) : 0.f;
+#pragma unroll
+          for (int u = 0; u < TB; ++u) acc[u] += v[u];
         }
-        if (n_ok) {
+      }
+      if (p.mode == EPI_STORE) {
+        if (n < p.N) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c + j < p.M) outp[(size_t)(c + j) * p.ldo] = v[j];
+          for (int u = 0; u < TB; ++u)
+            if (tok0 + u < t1) p.out[(size_t)(tok0 + u) * p.ldo + n] = acc[u];
+        }
+      } else if (p.splits > 1) {
+#pragma unroll
+        for (int u = 0; u < TB; ++u)                           // own slice of own buffer: nobody else reads it
+          if (tok0 + u < t1) red[(tok0 + u) * TC_BLOCK_N + fr] = acc[u];
+      }
+    }
+    if (p.mode != EPI_STORE) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");           // the four epilogue warps
+      if (p.mode == EPI_SWIGLU) {
+        const int f = tile * 64 + fr;
+        if (fr < 64 && f < p.F) {
+          for (int tok = t0; tok < t1; ++tok) {
+            const float g = red[tok * TC_BLOCK_N + fr], u = red[tok * TC_BLOCK_N + fr + 64];
+            p.hf[(size_t)tok * p.F + f] = f2bf(g / (1.0f + __expf(-g)) * u);
+          }
+        }
+      } else if (n < p.N) {                                    // EPI_QKV
+        const int head = n / p.D, dd = n - head * p.D, half = p.D >> 1;
+        const int C = *p.len_ptr;
+        const bool lo = dd < half;
+        const int j = lo ? dd : dd - half;
+        const int partner = lo ? fr + half : fr - half;
+        const bool rot = head < p.H + p.H_kv;
+        bf16* dst;                                             // element (row 0 / slot C) of this feature
+        size_t stride;
+        if (head < p.H) {
+          dst = p.q + (size_t)head * p.D + dd;
+          stride = (size_t)p.H * p.D;
+        } else if (rot) {
+          dst = p.kc + ((size_t)(head - p.H) * p.C_max + C) * p.D + dd;
+          stride = p.D;
+        } else {
+          dst = p.vc + ((size_t)(head - p.H - p.H_kv) * p.C_max + C) * p.D + dd;
+          stride = p.D;
+        }
+        const int t_end = head < p.H ? t1 : min(t1, p.C_max - C);      // never write past the cache
+        for (int tok0 = t0; tok0 < t_end; tok0 += TB) {
+          float2 cs[TB];
+#pragma unroll
+          for (int u = 0; u < TB; ++u) {
+            cs[u] = make_float2(1.f, 0.f);
+            if (rot && tok0 + u < t_end) cs[u] = p.rope_tab[(size_t)p.pos[tok0 + u] * half + j];
+          }
+#pragma unroll
+          for (int u = 0; u < TB; ++u) {
+            if (tok0 + u < t_end) {
+              const float v = red[(tok0 + u) * TC_BLOCK_N + fr], w = red[(tok0 + u) * TC_BLOCK_N + partner];
+              const float r = lo ? v * cs[u].x - w * cs[u].y : v * cs[u].x + w * cs[u].y;
+              dst[(size_t)(tok0 + u) * stride] = f2bf(r);
+            }
+          }
         }
       }
     }
   }
-  tc_fence_before();
-  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();                                          // nobody leaves while its buffer may be read
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
                  : "memory");
   }
-}
-
-// Y[m][n] = sum over splits, in split order.
-__global__ void k_reduce_splits(const float* __restrict__ part, float* __restrict__ y, size_t n, int splits) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  float acc = part[i];
-  for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
-  y[i] = acc;
 }
 
 }  // namespace bita

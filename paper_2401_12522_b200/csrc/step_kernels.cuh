@@ -1,6 +1,8 @@
-// Element-wise and integer kernels of one decoding pass: embedding/packing, RMSNorm,
-// rotary embedding + cache write, SwiGLU, argmax/top-k selection, the greedy
-// verification walk, next-tree construction and cache compaction.
+// Element-wise and integer kernels of one decoding pass: embedding/packing, RMSNorm (+ residual
+// add), argmax/top-k selection, the greedy verification walk, next-tree construction and cache
+// compaction.  (Rotary embedding, the cache write and SwiGLU live in the projection epilogues.)
+// Every kernel starts with the programmatic-dependent-launch pair: release the next kernel's
+// prologue, then wait for the predecessors before touching memory.
 #pragma once
 
 #include "common.cuh"
@@ -16,6 +18,8 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
                         const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
                         const bf16* __restrict__ mask_emb, int d, int V, float* __restrict__ x,
                         int32_t* __restrict__ pos, int32_t* __restrict__ row_token) {
+  pdl_launch();
+  pdl_wait();
   const int r = blockIdx.x;
   const int kind = plan.row_kind[r];
   const int idx = plan.row_idx[r];
@@ -38,6 +42,8 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
 // RMSNorm: xn = x * g / sqrt(mean(x^2) + eps), fp32 in, bf16 out.  One block per row.
 __global__ void k_rmsnorm(const float* __restrict__ x, const bf16* __restrict__ g, int d, float eps,
                           bf16* __restrict__ xn) {
+  pdl_launch();
+  pdl_wait();
   __shared__ float red[32];
   const int r = blockIdx.x;
   const float* xr = x + (size_t)r * d;
@@ -57,66 +63,19 @@ __global__ void k_rmsnorm(const float* __restrict__ x, const bf16* __restrict__ 
   for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
 }
 
-// ---------------------------------------------------------------------------------------------
-// Rotary embedding (half-split pairing: dims j and j + D/2) at the row's position id, then
-// q -> bf16 [M][H][D], k/v -> cache slot C + r of layout [H_kv][C_max][D].
-// rope_tab: float2 (cos, sin) [positions][D/2], computed in double on the host.
-// qkv: fp32 [nsplit][M][(H + 2 H_kv) D] split-K partials, summed here in split order.
-__global__ void k_rope_kv(const float* __restrict__ qkv, int nsplit, size_t split_stride,
-                          const int32_t* __restrict__ pos, const float2* __restrict__ rope_tab,
-                          const DevState* __restrict__ st, int H, int H_kv, int D, int C_max, bf16* __restrict__ q,
-                          bf16* __restrict__ kc, bf16* __restrict__ vc) {
-  const int r = blockIdx.x;
-  const int half = D >> 1;
-  const int p = pos[r];
-  const int slot = st->len + r;
-  const int nq = H * half, nk = H_kv * half;
-  const float* row = qkv + (size_t)r * (H + 2 * H_kv) * D;
-  auto ld = [&](const float* ptr) {
-    float acc = ptr[0];
-    for (int sp = 1; sp < nsplit; ++sp) acc += ptr[(size_t)sp * split_stride];
-    return acc;
-  };
-  for (int t = threadIdx.x; t < nq + nk; t += blockDim.x) {
-    const bool isq = t < nq;
-    const int u = isq ? t : t - nq;
-    const int h = u / half, j = u - h * half;
-    const float* src = row + (isq ? 0 : H * D) + h * D;
-    const float2 cs = rope_tab[(size_t)p * half + j];
-    const float a = ld(src + j), b = ld(src + j + half);
-    const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
-    if (isq) {
-      bf16* dst = q + ((size_t)r * H + h) * D;
-      dst[j] = f2bf(ra);
-      dst[j + half] = f2bf(rb);
-    } else if (slot < C_max) {
-      bf16* dst = kc + ((size_t)h * C_max + slot) * D;
-      dst[j] = f2bf(ra);
-      dst[j + half] = f2bf(rb);
-    }
-  }
-  if (slot < C_max) {
-    const float* vsrc = row + (H + H_kv) * D;
-    for (int t = threadIdx.x; t < H_kv * D; t += blockDim.x) {
-      const int h = t / D, j = t - h * D;
-      vc[((size_t)h * C_max + slot) * D + j] = f2bf(ld(vsrc + t));
-    }
-  }
-}
-
-// Residual add of split-K partials followed by the next RMSNorm:
-//   x[r] += sum_s part[s][r]   (split order);   xn[r] = x[r] * g / sqrt(mean(x[r]^2) + eps)  (bf16)
-// One block per row.
-__global__ void k_add_rmsnorm(float* __restrict__ x, const float* __restrict__ part, int nsplit, size_t split_stride,
-                              const bf16* __restrict__ g, int d, float eps, bf16* __restrict__ xn) {
+// Residual add followed by the next RMSNorm:
+//   x[r] += y[r];   xn[r] = x[r] * g / sqrt(mean(x[r]^2) + eps)  (bf16).   One block per row.
+__global__ void k_add_rmsnorm(float* __restrict__ x, const float* __restrict__ y, const bf16* __restrict__ g, int d,
+                              float eps, bf16* __restrict__ xn) {
+  pdl_launch();
+  pdl_wait();
   __shared__ float red[32];
   const int r = blockIdx.x;
   float* xr = x + (size_t)r * d;
-  const float* pr = part + (size_t)r * d;
+  const float* yr = y + (size_t)r * d;
   float ss = 0.f;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float v = xr[c];
-    for (int sp = 0; sp < nsplit; ++sp) v += pr[(size_t)sp * split_stride + c];
+    const float v = xr[c] + yr[c];
     xr[c] = v;
     ss += v * v;
   }
@@ -134,23 +93,6 @@ __global__ void k_add_rmsnorm(float* __restrict__ x, const float* __restrict__ p
   for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
 }
 
-// hf[r][f] = silu(gate) * up -> bf16, from the dual-tile projection output: fp32
-// [nsplit][M][ldg] where tile t holds gate features 64t..64t+63 in columns 128t..128t+63 and the
-// matching up features in columns 128t+64..128t+127.
-__global__ void k_swiglu(const float* __restrict__ gu, int nsplit, size_t split_stride, int ldg, int F, int M,
-                         bf16* __restrict__ hf) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)M * F) return;
-  const int r = (int)(i / F), f = (int)(i - (size_t)r * F);
-  const float* src = gu + (size_t)r * ldg + (f >> 6) * 128 + (f & 63);
-  float g = 0.f, u = 0.f;
-  for (int sp = 0; sp < nsplit; ++sp) {
-    g += src[(size_t)sp * split_stride];
-    u += src[(size_t)sp * split_stride + 64];
-  }
-  hf[i] = f2bf(g / (1.0f + __expf(-g)) * u);
-}
-
 // ---------------------------------------------------------------------------------------------
 // Argmax / sorted top-k of each logits row, order = (value descending, token id ascending).
 // One block per row; pass t picks the best entry strictly after the previous pick.
@@ -161,6 +103,8 @@ __device__ __forceinline__ bool before(float v1, int i1, float v2, int i2) {
 
 __global__ void k_select(DevPlan plan, const float* __restrict__ logits, int V, int32_t* __restrict__ sel_id,
                          float* __restrict__ sel_val) {
+  pdl_launch();
+  pdl_wait();
   __shared__ float sv[32];
   __shared__ int si[32];
   __shared__ float pv;
@@ -218,6 +162,8 @@ __global__ void k_select(DevPlan plan, const float* __restrict__ logits, int V, 
 // the last accepted candidate token").  One warp: lanes scan the children of the current node.
 __global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t* __restrict__ row_token,
                          const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec) {
+  pdl_launch();
+  pdl_wait();
   const int lane = threadIdx.x;
   const int N = plan.N;
   int cur = -1;
@@ -276,6 +222,8 @@ __global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t*
 // follows it drafts the first tree.  `last` = this is the final chunk of the query.
 __global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __restrict__ st,
                                  const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec, int last) {
+  pdl_launch();
+  pdl_wait();
   const int lane = threadIdx.x;
   const int C = st->len;
   const int T = chunk.n_query;
@@ -313,6 +261,8 @@ __global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __r
 // idx is increasing along a path.  grid = (L * H_kv), cache layout [L][H_kv][C_max][D].
 __global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, bf16* __restrict__ kc,
                           bf16* __restrict__ vc) {
+  pdl_launch();
+  pdl_wait();
   const int n_acc = rec->n_acc;
   if (n_acc == 0) return;
   const int C = rec->old_len;
@@ -333,11 +283,15 @@ __global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, b
 }
 
 __global__ void k_set_state(DevState* st, int len, int root) {
+  pdl_launch();
+  pdl_wait();
   if (threadIdx.x == 0) { st->len = len; st->root = root; }
   for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
 }
 
 __global__ void k_reset_state(DevState* st) {
+  pdl_launch();
+  pdl_wait();
   if (threadIdx.x == 0) { st->len = 0; st->root = -1; st->status = 0; st->pad = 0; }
   for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
 }
