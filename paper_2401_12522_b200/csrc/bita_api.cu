@@ -255,14 +255,19 @@ int make_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows) {
 struct GemmDesc {
   CUtensorMap a0, a1;
   int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
+  const void* w[2] = {nullptr, nullptr};   // the matrices themselves (for L2 prefetch by the previous projection)
+  size_t bytes = 0;                        // bytes of each
 };
 
 // Split-K factor (= cluster size): enough CTAs for about two per SM, at least 4 K blocks each.
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  int s = (296 + tiles / 2) / tiles;
+  // Clusters must be co-scheduled inside one GPC, so aim well below the 2 x 148 CTA slots.
+  int s = tiles >= 128 ? 1 : 256 / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
+  static const int cap = getenv("BITA_SPLIT_CAP") ? atoi(getenv("BITA_SPLIT_CAP")) : 8;
+  if (s > cap) s = cap;
   if (s > 8) s = 8;
   if (s < 1) s = 1;
   return s;
@@ -271,6 +276,9 @@ int gemm_splits(int tiles, int K, int max_splits) {
 int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
   g->K = K;
   g->dual = W1 ? 1 : 0;
+  g->w[0] = W0;
+  g->w[1] = W1;
+  g->bytes = (size_t)N * K * 2;
   int rc;
   if (W1) {           // N = rows of each of the two matrices
     g->tiles = (N + 63) / 64;
@@ -304,7 +312,7 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
-  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // reduction buffer
+  if ((size_t)stages * stage < (size_t)(M + 8) * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // reduction buffer
   p.stages = stages;
   const size_t smem = stages * stage + 1024;
   return launch(stream, pdl, dim3(g.tiles, g.splits), dim3(TC_THREADS), smem, (unsigned)g.splits, k_gemm_tc, g.a0,
@@ -335,7 +343,7 @@ int attn_splits(int H, int B, int M) {
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; float* tmp; bf16* hf; float* logits;
   int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
-  float2* rope_tab; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
+  float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
 };
 
@@ -364,6 +372,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
+  t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
   t.rec = (DevRecord*)take(sizeof(DevRecord));
   t.plan_step = take(PLAN_REGION_BYTES);
@@ -423,7 +432,8 @@ struct Timed {
 };
 
 // Projection of the first M rows of an activation buffer (BITA_MAX_ROWS rows allocated).
-int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
+int gemm(bita_ctx* c, const GemmDesc& g, const GemmDesc* next, const bf16* X, int M, GemmTcParams p) {
+  (void)next;
   const int n_pad = pad16(M);
   auto key = std::make_tuple((const void*)X, g.K, n_pad);
   auto it = c->act_maps.find(key);
@@ -482,7 +492,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   int rc;
   if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_embed, P, (const DevState*)b.state, tree_dev,
                    (const int32_t*)b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb, m.d, m.V, b.x,
-                   b.pos, b.row_token)))
+                   b.pos, b.row_token, (const float2*)b.rope_tab, m.D / 2, b.rope_blk)))
     return rc;
   if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_rmsnorm, (const float*)b.x, (const bf16*)c->g_attn[0], m.d,
                    m.rms_eps, b.xn)))
@@ -493,9 +503,9 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
     {   // q, k, v projection + rotary embedding + cache write
       GemmTcParams p{};
-      p.mode = EPI_QKV; p.q = b.q; p.kc = kc; p.vc = vc; p.pos = b.pos; p.rope_tab = b.rope_tab;
+      p.mode = EPI_QKV; p.q = b.q; p.kc = kc; p.vc = vc; p.rope_blk = b.rope_blk;
       p.len_ptr = &b.state->len; p.H = m.H; p.H_kv = m.H_kv; p.D = m.D; p.C_max = kv->C_max;
-      if ((rc = gemm(c, c->d_qkv[l], b.xn, M, p))) return rc;
+      if ((rc = gemm(c, c->d_qkv[l], &c->d_o[l], b.xn, M, p))) return rc;
     }
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
@@ -506,16 +516,17 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
       Timed t(c, 1);
       if ((rc = launch_attention(a, pdl, s))) return rc;
     }
-    if ((rc = gemm(c, c->d_o[l], b.att, M, epi_store(b.tmp, m.d)))) return rc;
+    if ((rc = gemm(c, c->d_o[l], &c->d_gu[l], b.att, M, epi_store(b.tmp, m.d)))) return rc;
     if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp,
                      (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn)))
       return rc;
     {   // gate/up projection + SwiGLU
       GemmTcParams p{};
       p.mode = EPI_SWIGLU; p.hf = b.hf; p.F = m.F;
-      if ((rc = gemm(c, c->d_gu[l], b.xn, M, p))) return rc;
+      if ((rc = gemm(c, c->d_gu[l], &c->d_dn[l], b.xn, M, p))) return rc;
     }
-    if ((rc = gemm(c, c->d_dn[l], b.hf, M, epi_store(b.tmp, m.d)))) return rc;
+    const GemmDesc* after_dn = l + 1 < m.L ? &c->d_qkv[l + 1] : (want_logits ? &c->d_head : nullptr);
+    if ((rc = gemm(c, c->d_dn[l], after_dn, b.hf, M, epi_store(b.tmp, m.d)))) return rc;
     const bf16* g_next = (const bf16*)(l + 1 < m.L ? c->g_attn[l + 1] : c->g_final);
     if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp, g_next, m.d,
                      m.rms_eps, b.xn)))
@@ -526,7 +537,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
                              cudaMemcpyDeviceToDevice, s));
   }
   if (want_logits) {
-    if ((rc = gemm(c, c->d_head, b.xn, M, epi_store(b.logits, m.V)))) return rc;
+    if ((rc = gemm(c, c->d_head, nullptr, b.xn, M, epi_store(b.logits, m.V)))) return rc;
     if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select, P, (const float*)b.logits, m.V, b.sel_id, b.sel_val)))
       return rc;
     c->launches += 1;

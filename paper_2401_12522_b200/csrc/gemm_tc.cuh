@@ -9,11 +9,11 @@
 // blocks (split-K); it streams its weight tiles through a ring of TMA-filled, 128-byte-swizzled
 // shared-memory stages, one elected thread issues tcgen05.mma into a TMEM accumulator, and four
 // epilogue warps read the accumulator back with tcgen05.ld.  The splits of one tile form a
-// thread-block cluster: every split parks its partial tile in its own shared memory, and after a
-// cluster barrier each split sums a slice of the rows over all partners through distributed shared
-// memory, always in split order - every output is a fixed-order sum (deterministic, and
-// independent of how many other rows the block holds) and no partial result ever goes to HBM.
-// The reducing thread then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
+// thread-block cluster: each split owns a slice of the block's rows, every split sends its partial
+// values for a row to the owner's shared memory (distributed shared memory stores), and after one
+// cluster barrier each owner sums its rows over the splits, always in split order - every output
+// is a fixed-order sum (deterministic, and independent of how many other rows the block holds)
+// and no partial result ever goes to HBM.  The owner then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
 // builds the 128-row weight tile from 64 gate rows and the 64 matching up rows, so both halves of
 // a product sit in the same tile); or rotary embedding with the q rows going to a bf16 buffer and
 // the k/v rows straight into the KV cache.
@@ -64,8 +64,7 @@ struct GemmTcParams {
   bf16* q;               // bf16 [M][H][D]
   bf16* kc;              // this layer's key cache   [H_kv][C_max][D]
   bf16* vc;              // this layer's value cache
-  const int32_t* pos;    // position id of each row
-  const float2* rope_tab;  // (cos, sin) [position][D/2]
+  const float2* rope_blk;  // (cos, sin) [row][D/2] for the block's position ids
   const int32_t* len_ptr;  // cache length C (device)
   int32_t H, H_kv, D, C_max;
 };
@@ -163,6 +162,11 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
@@ -191,10 +195,8 @@ __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float dsmem_ld(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void dsmem_st(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -239,6 +241,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   const uint32_t tmem_base = tmem_base_slot;
 
   if (threadIdx.x == 0) pdl_launch();          // the next kernel may start its prologue
+  if (threadIdx.x == 32) {                     // warm the descriptor cache while the barriers are set up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a0) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    if (p.dual) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a1) : "memory");
+  }
 
   if (warp == 0) {
     // ---------------- TMA producer
@@ -306,16 +313,29 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
   }
 
-  // ---------------- epilogue, part 1: this split's partial tile TMEM -> shared memory
-  // red[token][feature] (fp32) reuses the pipeline stages: every copy has landed and every MMA has
-  // read its operands once the accumulator barrier has completed.
+  // ---------------- epilogue, part 1: scatter this split's partial tile to the splits that own the rows
+  // Split r of the cluster owns rows [r * per, (r + 1) * per) of the block.  Its buffer (the
+  // pipeline stages, free once the accumulator barrier has completed) is laid out
+  // [source split][row within slice][128 features] fp32.  Every split writes its partial values
+  // for a row into the owner's buffer through distributed shared memory; after one cluster
+  // barrier each owner sums its rows over the source splits, in split order, from local memory.
   float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
   const int lg = warp & 3;                                     // TMEM lane group this warp may read
   const int fr = lg * 32 + lane;                               // feature row of the tile owned by this thread
+  const int per = (p.M + p.splits - 1) / p.splits;             // rows per owner
+  const int rank = p.splits > 1 ? (int)cluster_rank() : 0;
+  bool acc_ok = true;
   if (warp >= 2) {
-    bool ok = true;
-    if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
+    if (nkb > 0) acc_ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     tc_fence_after();
+  }
+  // A partner may only write into this CTA's stages once this CTA's own pipeline has drained.
+  __syncwarp();
+  if (p.splits > 1) cluster_sync_all();
+  if (warp >= 2) {
+    const bool ok = acc_ok;
+    int owner = 0, owner_end = per;
+    uint32_t obase = (p.splits > 1 ? dsmem_addr(smem_base, 0u) : smem_base) + (uint32_t)(rank * per * TC_BLOCK_N + fr) * 4u;
     for (int c = 0; c < p.n_pad; c += 16) {
       float v[16];
       if (nkb > 0 && ok) {
@@ -325,107 +345,99 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         for (int j = 0; j < 16; ++j) v[j] = 0.f;
       }
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (c + j < p.M) red[(c + j) * TC_BLOCK_N + fr] = v[j];
+      for (int j = 0; j < 16; ++j) {
+        const int tok = c + j;
+        if (tok < p.M) {
+          if (tok >= owner_end) {
+            ++owner;
+            owner_end += per;
+            obase = dsmem_addr(smem_base, (uint32_t)owner) + (uint32_t)(rank * per * TC_BLOCK_N + fr) * 4u;
+          }
+          dsmem_st(obase + (uint32_t)((tok - owner * per) * TC_BLOCK_N) * 4u, v[j]);
+        }
+      }
     }
   }
   tc_fence_before();
   __syncwarp();
-  cluster_sync_all();                                          // partial tiles of all splits are in place
+  if (p.splits > 1) cluster_sync_all();                        // every partial value has reached its owner
+  else __syncthreads();
 
-  // ---------------- epilogue, part 2: each split reduces a slice of the rows over all splits, in
-  // split order, and applies the fused operation.  Rows are handled eight at a time so that the
-  // (remote) shared-memory and global loads of a batch are in flight together.
+  // ---------------- epilogue, part 2: owner-side reduction (local) + fused operation.
+  // A thread handles 4 consecutive features (quad = lane) of one row at a time; the four warps
+  // take rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 features
+  // (16 lanes) away, so they are exchanged with a warp shuffle.
   if (warp >= 2) {
-    constexpr int TB = 8;
     pdl_wait();
-    const int rank = (int)cluster_rank();
-    const int per = (p.M + p.splits - 1) / p.splits;
-    const int t0 = rank * per, t1 = min(p.M, t0 + per);
-    const uint32_t red_u32 = smem_base;
-    const int n = tile * TC_BLOCK_N + fr;                      // output feature (EPI_STORE / EPI_QKV)
-    for (int tok0 = t0; tok0 < t1; tok0 += TB) {
-      float acc[TB];
-#pragma unroll
-      for (int u = 0; u < TB; ++u) acc[u] = 0.f;
-      if (p.splits == 1) {
-#pragma unroll
-        for (int u = 0; u < TB; ++u)
-          if (tok0 + u < t1) acc[u] = red[(tok0 + u) * TC_BLOCK_N + fr];
-      } else {
-        for (int r = 0; r < p.splits; ++r) {
-          const uint32_t base = dsmem_addr(red_u32, (uint32_t)r) + (uint32_t)fr * 4u;
-          float v[TB];
-#pragma unroll
-          for (int u = 0; u < TB; ++u)
-            v[u] = (tok0 + u < t1) ? dsmem_ld(base + (uint32_t)((tok0 + u) * TC_BLOCK_N) * 4u) : 0.f;
-#pragma unroll
-          for (int u = 0; u < TB; ++u) acc[u] += v[u];
-        }
+    const int t0 = rank * per, cnt = min(p.M, t0 + per) - t0;  // rows owned by this split
+    const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
+    const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
+    for (int tl = warp - 2; tl < cnt; tl += 4) {
+      const int tok = t0 + tl;
+      float4 acc = *reinterpret_cast<const float4*>(red + (size_t)tl * TC_BLOCK_N + 4 * lane);
+      for (int r = 1; r < p.splits; ++r) {
+        const float4 v = *reinterpret_cast<const float4*>(red + (size_t)(r * per + tl) * TC_BLOCK_N + 4 * lane);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
       }
       if (p.mode == EPI_STORE) {
-        if (n < p.N) {
-#pragma unroll
-          for (int u = 0; u < TB; ++u)
-            if (tok0 + u < t1) p.out[(size_t)(tok0 + u) * p.ldo + n] = acc[u];
-        }
-      } else if (p.splits > 1) {
-#pragma unroll
-        for (int u = 0; u < TB; ++u)                           // own slice of own buffer: nobody else reads it
-          if (tok0 + u < t1) red[(tok0 + u) * TC_BLOCK_N + fr] = acc[u];
-      }
-    }
-    if (p.mode != EPI_STORE) {
-      asm volatile("bar.sync 1, 128;" ::: "memory");           // the four epilogue warps
-      if (p.mode == EPI_SWIGLU) {
-        const int f = tile * 64 + fr;
-        if (fr < 64 && f < p.F) {
-          for (int tok = t0; tok < t1; ++tok) {
-            const float g = red[tok * TC_BLOCK_N + fr], u = red[tok * TC_BLOCK_N + fr + 64];
-            p.hf[(size_t)tok * p.F + f] = f2bf(g / (1.0f + __expf(-g)) * u);
-          }
-        }
-      } else if (n < p.N) {                                    // EPI_QKV
-        const int head = n / p.D, dd = n - head * p.D, half = p.D >> 1;
-        const int C = *p.len_ptr;
-        const bool lo = dd < half;
-        const int j = lo ? dd : dd - half;
-        const int partner = lo ? fr + half : fr - half;
-        const bool rot = head < p.H + p.H_kv;
-        bf16* dst;                                             // element (row 0 / slot C) of this feature
-        size_t stride;
-        if (head < p.H) {
-          dst = p.q + (size_t)head * p.D + dd;
-          stride = (size_t)p.H * p.D;
-        } else if (rot) {
-          dst = p.kc + ((size_t)(head - p.H) * p.C_max + C) * p.D + dd;
-          stride = p.D;
+        float* dst = p.out + (size_t)tok * p.ldo + n4;
+        if (n4 + 3 < p.N && (p.ldo & 3) == 0) {
+          *reinterpret_cast<float4*>(dst) = acc;
         } else {
-          dst = p.vc + ((size_t)(head - p.H - p.H_kv) * p.C_max + C) * p.D + dd;
-          stride = p.D;
+          if (n4 < p.N) dst[0] = acc.x;
+          if (n4 + 1 < p.N) dst[1] = acc.y;
+          if (n4 + 2 < p.N) dst[2] = acc.z;
+          if (n4 + 3 < p.N) dst[3] = acc.w;
         }
-        const int t_end = head < p.H ? t1 : min(t1, p.C_max - C);      // never write past the cache
-        for (int tok0 = t0; tok0 < t_end; tok0 += TB) {
-          float2 cs[TB];
-#pragma unroll
-          for (int u = 0; u < TB; ++u) {
-            cs[u] = make_float2(1.f, 0.f);
-            if (rot && tok0 + u < t_end) cs[u] = p.rope_tab[(size_t)p.pos[tok0 + u] * half + j];
+      } else if (p.mode == EPI_SWIGLU) {
+        // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
+        const float ux = __shfl_down_sync(0xffffffffu, acc.x, 16), uy = __shfl_down_sync(0xffffffffu, acc.y, 16);
+        const float uz = __shfl_down_sync(0xffffffffu, acc.z, 16), uw = __shfl_down_sync(0xffffffffu, acc.w, 16);
+        const int f = tile * 64 + 4 * lane;
+        if (lane < 16 && f < p.F) {                            // F is a multiple of 8: a quad is all in or all out
+          const float h0 = acc.x / (1.0f + __expf(-acc.x)) * ux, h1 = acc.y / (1.0f + __expf(-acc.y)) * uy;
+          const float h2 = acc.z / (1.0f + __expf(-acc.z)) * uz, h3 = acc.w / (1.0f + __expf(-acc.w)) * uw;
+          uint2 pk;
+          pk.x = pack_bf16x2(h0, h1);
+          pk.y = pack_bf16x2(h2, h3);
+          *reinterpret_cast<uint2*>(p.hf + (size_t)tok * p.F + f) = pk;
+        }
+      } else {                                                 // EPI_QKV
+        const int half = p.D >> 1;
+        const int sh = half >> 2;                              // partner quad is `sh` lanes away (16 or 8)
+        // partner values: the other half of the same head
+        const float wx = __shfl_xor_sync(0xffffffffu, acc.x, sh), wy = __shfl_xor_sync(0xffffffffu, acc.y, sh);
+        const float wz = __shfl_xor_sync(0xffffffffu, acc.z, sh), ww = __shfl_xor_sync(0xffffffffu, acc.w, sh);
+        if (n4 < p.N) {                                        // N is a multiple of D: a quad is all in or all out
+          const int head = n4 / p.D, dd = n4 - head * p.D;
+          const bool lo = dd < half;
+          const int j = lo ? dd : dd - half;
+          float4 r = acc;
+          if (head < p.H + p.H_kv) {
+            const float4 c01 = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + j);
+            const float4 c23 = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + j + 2);
+            const float sg = lo ? -1.f : 1.f;
+            r.x = acc.x * c01.x + sg * wx * c01.y;
+            r.y = acc.y * c01.z + sg * wy * c01.w;
+            r.z = acc.z * c23.x + sg * wz * c23.y;
+            r.w = acc.w * c23.z + sg * ww * c23.w;
           }
-#pragma unroll
-          for (int u = 0; u < TB; ++u) {
-            if (tok0 + u < t_end) {
-              const float v = red[(tok0 + u) * TC_BLOCK_N + fr], w = red[(tok0 + u) * TC_BLOCK_N + partner];
-              const float r = lo ? v * cs[u].x - w * cs[u].y : v * cs[u].x + w * cs[u].y;
-              dst[(size_t)(tok0 + u) * stride] = f2bf(r);
-            }
+          uint2 pk;
+          pk.x = pack_bf16x2(r.x, r.y);
+          pk.y = pack_bf16x2(r.z, r.w);
+          const int slot = C + tok;
+          if (head < p.H) {
+            *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
+          } else if (slot < p.C_max) {
+            bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
+                                             : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
+            *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
           }
         }
       }
     }
   }
-  __syncwarp();
-  cluster_sync_all();                                          // nobody leaves while its buffer may be read
+  __syncthreads();
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)

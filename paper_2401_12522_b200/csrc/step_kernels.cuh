@@ -17,7 +17,8 @@ namespace bita {
 __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int32_t* __restrict__ tree_tokens,
                         const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
                         const bf16* __restrict__ mask_emb, int d, int V, float* __restrict__ x,
-                        int32_t* __restrict__ pos, int32_t* __restrict__ row_token) {
+                        int32_t* __restrict__ pos, int32_t* __restrict__ row_token,
+                        const float2* __restrict__ rope_tab, int half, float2* __restrict__ rope_blk) {
   pdl_launch();
   pdl_wait();
   const int r = blockIdx.x;
@@ -36,6 +37,9 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
   }
   float* xr = x + (size_t)r * d;
   for (int c = threadIdx.x; c < d; c += blockDim.x) xr[c] = src ? bf2f(src[c]) : 0.0f;
+  // (cos, sin) row of this row's position id, for the rotary embedding in the q/k/v projection
+  const int p = st->len + plan.rel_pos[r];
+  for (int j = threadIdx.x; j < half; j += blockDim.x) rope_blk[(size_t)r * half + j] = rope_tab[(size_t)p * half + j];
 }
 
 // ---------------------------------------------------------------------------------------------
