@@ -341,7 +341,7 @@ int attn_splits(int H, int B, int M) {
 
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
-  float* x; bf16* xn; bf16* q; bf16* att; float* tmp; bf16* hf; float* logits;
+  float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
   int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
@@ -361,7 +361,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.xn = (bf16*)take(R * wide * 2);
   t.q = (bf16*)take(R * m.H * m.D * 2);
   t.att = (bf16*)take(R * m.H * m.D * 2);
-  t.tmp = (float*)take(R * (size_t)m.d * 4);
+  t.sumsq = (unsigned long long*)take((size_t)(2 * m.L + 1) * R * 8);
   t.hf = (bf16*)take(R * (size_t)m.F * 2);
   t.logits = (float*)take(R * (size_t)m.V * 4);
   t.sel_id = (int32_t*)take(R * BITA_MAX_TOPK * 4);
@@ -432,8 +432,7 @@ struct Timed {
 };
 
 // Projection of the first M rows of an activation buffer (BITA_MAX_ROWS rows allocated).
-int gemm(bita_ctx* c, const GemmDesc& g, const GemmDesc* next, const bf16* X, int M, GemmTcParams p) {
-  (void)next;
+int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   const int n_pad = pad16(M);
   auto key = std::make_tuple((const void*)X, g.K, n_pad);
   auto it = c->act_maps.find(key);
@@ -490,22 +489,33 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
   const bool pdl = c->pdl;
   int rc;
+  const int n_slots = 2 * m.L + 1;
+  auto slot = [&](int i) { return b.sumsq + (size_t)i * BITA_MAX_ROWS; };
   if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_embed, P, (const DevState*)b.state, tree_dev,
                    (const int32_t*)b.query_tokens, (const bf16*)c->tok_emb, (const bf16*)c->mask_emb, m.d, m.V, b.x,
-                   b.pos, b.row_token, (const float2*)b.rope_tab, m.D / 2, b.rope_blk)))
+                   b.pos, b.row_token, (const float2*)b.rope_tab, m.D / 2, b.rope_blk, (const bf16*)c->g_attn[0],
+                   b.xn, b.sumsq, n_slots)))
     return rc;
-  if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_rmsnorm, (const float*)b.x, (const bf16*)c->g_attn[0], m.d,
-                   m.rms_eps, b.xn)))
-    return rc;
-  c->launches += 2;
+  c->launches += 1;
+  auto with_norm = [&](GemmTcParams p, int in_slot) {
+    p.in_sumsq = slot(in_slot);
+    p.norm_d = m.d;
+    p.norm_eps = m.rms_eps;
+    return p;
+  };
+  auto epi_resid = [&](const void* gain, int out_slot) {
+    GemmTcParams p{};
+    p.mode = EPI_RESID; p.x = b.x; p.xhat = b.xn; p.gain = (const bf16*)gain; p.out_sumsq = slot(out_slot);
+    return p;
+  };
   for (int l = 0; l < m.L; ++l) {
     bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
     bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
-    {   // q, k, v projection + rotary embedding + cache write
+    {   // attention RMSNorm scale + q, k, v projection + rotary embedding + cache write
       GemmTcParams p{};
       p.mode = EPI_QKV; p.q = b.q; p.kc = kc; p.vc = vc; p.rope_blk = b.rope_blk;
       p.len_ptr = &b.state->len; p.H = m.H; p.H_kv = m.H_kv; p.D = m.D; p.C_max = kv->C_max;
-      if ((rc = gemm(c, c->d_qkv[l], &c->d_o[l], b.xn, M, p))) return rc;
+      if ((rc = gemm(c, c->d_qkv[l], b.xn, M, with_norm(p, 2 * l)))) return rc;
     }
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
@@ -516,28 +526,23 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
       Timed t(c, 1);
       if ((rc = launch_attention(a, pdl, s))) return rc;
     }
-    if ((rc = gemm(c, c->d_o[l], &c->d_gu[l], b.att, M, epi_store(b.tmp, m.d)))) return rc;
-    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp,
-                     (const bf16*)c->g_ffn[l], m.d, m.rms_eps, b.xn)))
-      return rc;
-    {   // gate/up projection + SwiGLU
+    c->launches += 2;
+    // output projection + residual add; leaves x * g_ffn and the row statistics for the FFN norm
+    if ((rc = gemm(c, c->d_o[l], b.att, M, epi_resid(c->g_ffn[l], 2 * l + 1)))) return rc;
+    {   // FFN RMSNorm scale + gate/up projection + SwiGLU
       GemmTcParams p{};
       p.mode = EPI_SWIGLU; p.hf = b.hf; p.F = m.F;
-      if ((rc = gemm(c, c->d_gu[l], &c->d_dn[l], b.xn, M, p))) return rc;
+      if ((rc = gemm(c, c->d_gu[l], b.xn, M, with_norm(p, 2 * l + 1)))) return rc;
     }
-    const GemmDesc* after_dn = l + 1 < m.L ? &c->d_qkv[l + 1] : (want_logits ? &c->d_head : nullptr);
-    if ((rc = gemm(c, c->d_dn[l], after_dn, b.hf, M, epi_store(b.tmp, m.d)))) return rc;
-    const bf16* g_next = (const bf16*)(l + 1 < m.L ? c->g_attn[l + 1] : c->g_final);
-    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_add_rmsnorm, b.x, (const float*)b.tmp, g_next, m.d,
-                     m.rms_eps, b.xn)))
-      return rc;
-    c->launches += 4;
+    // down projection + residual add; leaves x * gain of the next norm (next layer's or the final one)
+    const void* g_next = l + 1 < m.L ? c->g_attn[l + 1] : c->g_final;
+    if ((rc = gemm(c, c->d_dn[l], b.hf, M, epi_resid(g_next, 2 * l + 2)))) return rc;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)l * BITA_MAX_ROWS * m.d, b.x, (size_t)M * m.d * 4,
                              cudaMemcpyDeviceToDevice, s));
   }
   if (want_logits) {
-    if ((rc = gemm(c, c->d_head, nullptr, b.xn, M, epi_store(b.logits, m.V)))) return rc;
+    if ((rc = gemm(c, c->d_head, b.xn, M, with_norm(epi_store(b.logits, m.V), 2 * m.L)))) return rc;
     if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select, P, (const float*)b.logits, m.V, b.sel_id, b.sel_val)))
       return rc;
     c->launches += 1;

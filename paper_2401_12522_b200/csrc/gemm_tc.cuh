@@ -41,7 +41,23 @@ enum GemmEpilogue : int32_t {
   EPI_STORE = 0,    // out[m][n] = y                                   (fp32)
   EPI_SWIGLU = 1,   // dual tile: hf[m][f] = silu(gate) * up            (bf16)
   EPI_QKV = 2,      // rotary embedding, q -> bf16 buffer, k/v -> cache (bf16)
+  EPI_RESID = 3,    // x[m][n] += y; xhat = bf16(x * gain); row sums of x^2 for the next RMSNorm
 };
+
+// RMSNorm is split between producer and consumer so that it needs no pass of its own: the
+// projection that updates the residual stream x also writes xhat = bf16(x * gain) and adds its
+// tile's share of sum(x^2) per row into a fixed-point accumulator (integer atomics: the sum does
+// not depend on arrival order); the projection that consumes xhat multiplies its result by
+// rstd = 1 / sqrt(sum / d + eps) per row, which is the same thing since the projection is linear.
+constexpr float SUMSQ_SCALE = 268435456.0f;      // 2^28 fixed-point units per 1.0
+
+__device__ __forceinline__ float rstd_from_sumsq(unsigned long long fx, int d, float eps) {
+  const float ss = (float)((double)fx * (1.0 / 268435456.0));
+  return rsqrtf(ss / (float)d + eps);
+}
+__device__ __forceinline__ unsigned long long sumsq_to_fixed(float v) {
+  return __double2ull_rn((double)v * 268435456.0);
+}
 
 struct GemmTcParams {
   int32_t M;             // valid rows of X
@@ -54,12 +70,21 @@ struct GemmTcParams {
   int32_t tmem_cols;     // power of two >= max(32, n_pad)
   int32_t mode;          // GemmEpilogue
   int32_t* status;       // device status word (sticky error flag)
+  // row scale of the input (RMSNorm statistics of the rows of X), or null: y *= rstd(row)
+  const unsigned long long* in_sumsq;
+  int32_t norm_d;
+  float norm_eps;
   // EPI_STORE
   float* out;            // fp32 [M][ldo]
   int32_t ldo;
   // EPI_SWIGLU
   bf16* hf;              // bf16 [M][F]
   int32_t F;
+  // EPI_RESID
+  float* x;              // fp32 [M][N] residual stream, updated in place
+  bf16* xhat;            // bf16 [M][N] = x * gain
+  const bf16* gain;      // bf16 [N] gain of the RMSNorm that follows
+  unsigned long long* out_sumsq;   // [M] fixed-point sum of x^2 per row (zeroed by the pass's first kernel)
   // EPI_QKV
   bf16* q;               // bf16 [M][H][D]
   bf16* kc;              // this layer's key cache   [H_kv][C_max][D]
@@ -372,6 +397,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     const int t0 = rank * per, cnt = min(p.M, t0 + per) - t0;  // rows owned by this split
     const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
     const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
+    float g4[4] = {1.f, 1.f, 1.f, 1.f};
+    if (p.mode == EPI_RESID && n4 + 3 < p.N) {
+      const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
+      const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.x));
+      const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
+      g4[0] = a.x; g4[1] = a.y; g4[2] = b.x; g4[3] = b.y;
+    }
     for (int tl = warp - 2; tl < cnt; tl += 4) {
       const int tok = t0 + tl;
       float4 acc = *reinterpret_cast<const float4*>(red + (size_t)tl * TC_BLOCK_N + 4 * lane);
@@ -379,7 +411,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         const float4 v = *reinterpret_cast<const float4*>(red + (size_t)(r * per + tl) * TC_BLOCK_N + 4 * lane);
         acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
       }
-      if (p.mode == EPI_STORE) {
+      if (p.in_sumsq) {                                        // the input rows were left unnormalised
+        const float rs = rstd_from_sumsq(p.in_sumsq[tok], p.norm_d, p.norm_eps);
+        acc.x *= rs; acc.y *= rs; acc.z *= rs; acc.w *= rs;
+      }
+      if (p.mode == EPI_RESID) {
+        float ss = 0.f;
+        if (n4 + 3 < p.N) {                                    // N (the model width) is a multiple of 8
+          float4* xp = reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4);
+          float4 xv = *xp;
+          xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
+          *xp = xv;
+          uint2 pk;
+          pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
+          pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
+          *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
+          ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) atomicAdd(p.out_sumsq + tok, sumsq_to_fixed(ss));
+      } else if (p.mode == EPI_STORE) {
         float* dst = p.out + (size_t)tok * p.ldo + n4;
         if (n4 + 3 < p.N && (p.ldo & 3) == 0) {
           *reinterpret_cast<float4*>(dst) = acc;

@@ -1,11 +1,13 @@
-// Element-wise and integer kernels of one decoding pass: embedding/packing, RMSNorm (+ residual
-// add), argmax/top-k selection, the greedy verification walk, next-tree construction and cache
-// compaction.  (Rotary embedding, the cache write and SwiGLU live in the projection epilogues.)
+// Element-wise and integer kernels of one decoding pass: embedding/packing, argmax/top-k
+// selection, the greedy verification walk, next-tree construction and cache compaction.
+// (Residual add, RMSNorm, rotary embedding, the cache write and SwiGLU live in the projection
+// epilogues.)
 // Every kernel starts with the programmatic-dependent-launch pair: release the next kernel's
 // prologue, then wait for the predecessors before touching memory.
 #pragma once
 
 #include "common.cuh"
+#include "gemm_tc.cuh"
 
 namespace bita {
 
@@ -18,7 +20,9 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
                         const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
                         const bf16* __restrict__ mask_emb, int d, int V, float* __restrict__ x,
                         int32_t* __restrict__ pos, int32_t* __restrict__ row_token,
-                        const float2* __restrict__ rope_tab, int half, float2* __restrict__ rope_blk) {
+                        const float2* __restrict__ rope_tab, int half, float2* __restrict__ rope_blk,
+                        const bf16* __restrict__ gain0, bf16* __restrict__ xhat,
+                        unsigned long long* __restrict__ sumsq, int n_slots) {
   pdl_launch();
   pdl_wait();
   const int r = blockIdx.x;
@@ -36,65 +40,29 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
     row_token[r] = (tok >= 0 && tok < V) ? tok : -1;
   }
   float* xr = x + (size_t)r * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) xr[c] = src ? bf2f(src[c]) : 0.0f;
+  bf16* hr = xhat + (size_t)r * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = src ? bf2f(src[c]) : 0.0f;
+    xr[c] = v;
+    hr[c] = f2bf(v * bf2f(gain0[c]));                     // input of the first projection: x * gain, unnormalised
+    ss += v * v;
+  }
+  // RMSNorm statistics: slot 0 is this row's sum of squares, the later slots are accumulated by
+  // the projections of the pass and start from zero
+  __shared__ float red[32];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    sumsq[r] = sumsq_to_fixed(t);
+  }
+  for (int sl = 1 + threadIdx.x; sl < n_slots; sl += blockDim.x) sumsq[(size_t)sl * BITA_MAX_ROWS + r] = 0ull;
   // (cos, sin) row of this row's position id, for the rotary embedding in the q/k/v projection
   const int p = st->len + plan.rel_pos[r];
   for (int j = threadIdx.x; j < half; j += blockDim.x) rope_blk[(size_t)r * half + j] = rope_tab[(size_t)p * half + j];
-}
-
-// ---------------------------------------------------------------------------------------------
-// RMSNorm: xn = x * g / sqrt(mean(x^2) + eps), fp32 in, bf16 out.  One block per row.
-__global__ void k_rmsnorm(const float* __restrict__ x, const bf16* __restrict__ g, int d, float eps,
-                          bf16* __restrict__ xn) {
-  pdl_launch();
-  pdl_wait();
-  __shared__ float red[32];
-  const int r = blockIdx.x;
-  const float* xr = x + (size_t)r * d;
-  float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) { float v = xr[c]; ss += v * v; }
-  ss = warp_sum(ss);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
-  }
-  __syncthreads();
-  const float inv = red[0];
-  bf16* o = xn + (size_t)r * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
-}
-
-// Residual add followed by the next RMSNorm:
-//   x[r] += y[r];   xn[r] = x[r] * g / sqrt(mean(x[r]^2) + eps)  (bf16).   One block per row.
-__global__ void k_add_rmsnorm(float* __restrict__ x, const float* __restrict__ y, const bf16* __restrict__ g, int d,
-                              float eps, bf16* __restrict__ xn) {
-  pdl_launch();
-  pdl_wait();
-  __shared__ float red[32];
-  const int r = blockIdx.x;
-  float* xr = x + (size_t)r * d;
-  const float* yr = y + (size_t)r * d;
-  float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float v = xr[c] + yr[c];
-    xr[c] = v;
-    ss += v * v;
-  }
-  ss = warp_sum(ss);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)d + eps);
-  }
-  __syncthreads();
-  const float inv = red[0];
-  bf16* o = xn + (size_t)r * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = f2bf(xr[c] * inv * bf2f(g[c]));
 }
 
 // ---------------------------------------------------------------------------------------------
