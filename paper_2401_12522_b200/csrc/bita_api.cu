@@ -259,18 +259,46 @@ struct GemmDesc {
   size_t bytes = 0;                        // bytes of each
 };
 
-// Split-K factor (= cluster size): enough CTAs for about two per SM, at least 4 K blocks each.
+// Split-K factor (= cluster size).  A kernel launched as clusters gets one CTA per SM and a
+// cluster-size-dependent number of clusters at a time (the runtime reports it), so a split is only
+// worth it when all its CTAs run in one wave; tile counts above the SM count run unsplit with two
+// CTAs per SM.
+int max_active_clusters(int cluster) {
+  static int cache[9] = {0};
+  if (cluster < 1 || cluster > 8) return 0;
+  if (!cache[cluster]) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(cluster * 32, cluster);
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = 200 * 1024;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1;
+    at[0].val.clusterDim.y = cluster;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+    if (cudaOccupancyMaxActiveClusters(&n, k_gemm_tc, &cfg) != cudaSuccess || n < 1) {
+      static const int fallback[9] = {0, 148, 74, 45, 33, 26, 22, 18, 15};   // what a B200 reported
+      n = fallback[cluster];
+      cudaGetLastError();
+    }
+    cache[cluster] = n;
+  }
+  return cache[cluster];
+}
+
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  // Clusters must be co-scheduled inside one GPC, so aim well below the 2 x 148 CTA slots.
-  int s = tiles >= 128 ? 1 : 256 / tiles;
-  if (s > kb / 4) s = kb / 4;
-  if (s > max_splits) s = max_splits;
   static const int cap = getenv("BITA_SPLIT_CAP") ? atoi(getenv("BITA_SPLIT_CAP")) : 8;
-  if (s > cap) s = cap;
-  if (s > 8) s = 8;
-  if (s < 1) s = 1;
-  return s;
+  int best = 1;
+  for (int s = 2; s <= 8 && s <= max_splits && s <= cap; ++s) {
+    if (kb / s < 4) break;
+    if (tiles <= max_active_clusters(s)) best = s;            // all tiles * s CTAs resident at once
+  }
+  return best;
 }
 
 int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
@@ -300,23 +328,29 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
                    cudaStream_t stream) {
   static bool attr_set = false;
   if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
     attr_set = true;
   }
-  p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.splits = g.splits; p.dual = g.dual;
+  int splits = g.splits;
+  p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.dual = g.dual;
   int cols = 32;
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
   const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  const size_t budget = (n_pad <= 96 ? 110 : 220) * 1024;       // two CTAs per SM while the block is small
+  // One wave with one CTA per SM gets the whole shared memory; more tiles than SMs share it two per SM.
+  const bool two_per_sm = splits == 1 && g.tiles > 148 && n_pad <= 96;
+  const size_t budget = (two_per_sm ? 110 : 220) * 1024;
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
-  if ((size_t)stages * stage < (size_t)(M + 8) * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // reduction buffer
+  // the epilogue reuses the stages for its staging and receive buffers
+  if ((size_t)stages * stage < ((size_t)2 * M + splits) * TC_BLOCK_N * 4) splits = 1;
+  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;
+  p.splits = splits;
   p.stages = stages;
   const size_t smem = stages * stage + 1024;
-  return launch(stream, pdl, dim3(g.tiles, g.splits), dim3(TC_THREADS), smem, (unsigned)g.splits, k_gemm_tc, g.a0,
-                g.a1, map_b, p);
+  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, (unsigned)splits, k_gemm_tc, g.a0, g.a1,
+                map_b, p);
 }
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }

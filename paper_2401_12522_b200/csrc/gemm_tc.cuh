@@ -233,6 +233,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t bar_empty[16];
   __shared__ __align__(8) uint64_t bar_acc;
   __shared__ uint32_t tmem_base_slot;
+  __shared__ float rstd_s[BITA_MAX_ROWS];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -338,29 +339,25 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
   }
 
-  // ---------------- epilogue, part 1: scatter this split's partial tile to the splits that own the rows
-  // Split r of the cluster owns rows [r * per, (r + 1) * per) of the block.  Its buffer (the
-  // pipeline stages, free once the accumulator barrier has completed) is laid out
-  // [source split][row within slice][128 features] fp32.  Every split writes its partial values
-  // for a row into the owner's buffer through distributed shared memory; after one cluster
-  // barrier each owner sums its rows over the source splits, in split order, from local memory.
-  float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
-  const int lg = warp & 3;                                     // TMEM lane group this warp may read
-  const int fr = lg * 32 + lane;                               // feature row of the tile owned by this thread
+  // ---------------- epilogue
+  // The pipeline stages are free once the accumulator barrier has completed; they are reused as
+  //   stg  [M][128] fp32           this split's partial tile, row-major
+  //   recv [splits][per][128] fp32 (splits > 1) partial values of the rows this split owns
+  // Split r of the cluster owns rows [r * per, (r + 1) * per).  Part 1 moves the accumulator to
+  // `stg` (thread = feature).  With splits > 1 every split then sends each row of `stg` to the
+  // row's owner as 16-byte distributed-shared-memory stores, and after one cluster barrier the
+  // owner sums its rows over the source splits, in split order, from local memory.
+  float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
   const int per = (p.M + p.splits - 1) / p.splits;             // rows per owner
   const int rank = p.splits > 1 ? (int)cluster_rank() : 0;
-  bool acc_ok = true;
+  const uint32_t recv_off = (uint32_t)p.M * TC_BLOCK_N * 4u;   // byte offset of `recv` from the buffer base
+  const float* recv = p.splits > 1 ? stg + (size_t)p.M * TC_BLOCK_N : stg;
   if (warp >= 2) {
-    if (nkb > 0) acc_ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
+    const int lg = warp & 3;                                   // TMEM lane group this warp may read
+    const int fr = lg * 32 + lane;                             // feature row of the tile owned by this thread
+    bool ok = true;
+    if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     tc_fence_after();
-  }
-  // A partner may only write into this CTA's stages once this CTA's own pipeline has drained.
-  __syncwarp();
-  if (p.splits > 1) cluster_sync_all();
-  if (warp >= 2) {
-    const bool ok = acc_ok;
-    int owner = 0, owner_end = per;
-    uint32_t obase = (p.splits > 1 ? dsmem_addr(smem_base, 0u) : smem_base) + (uint32_t)(rank * per * TC_BLOCK_N + fr) * 4u;
     for (int c = 0; c < p.n_pad; c += 16) {
       float v[16];
       if (nkb > 0 && ok) {
@@ -370,33 +367,42 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         for (int j = 0; j < 16; ++j) v[j] = 0.f;
       }
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const int tok = c + j;
-        if (tok < p.M) {
-          if (tok >= owner_end) {
-            ++owner;
-            owner_end += per;
-            obase = dsmem_addr(smem_base, (uint32_t)owner) + (uint32_t)(rank * per * TC_BLOCK_N + fr) * 4u;
-          }
-          dsmem_st(obase + (uint32_t)((tok - owner * per) * TC_BLOCK_N) * 4u, v[j]);
-        }
-      }
+      for (int j = 0; j < 16; ++j)
+        if (c + j < p.M) stg[(c + j) * TC_BLOCK_N + fr] = v[j];
     }
   }
   tc_fence_before();
-  __syncwarp();
-  if (p.splits > 1) cluster_sync_all();                        // every partial value has reached its owner
-  else __syncthreads();
+  __syncthreads();
+  if (p.splits > 1) {
+    // a partner may only write into this CTA's stages once this CTA's own pipeline has drained
+    cluster_sync_all();
+    for (int tok = warp; tok < p.M; tok += TC_THREADS / 32) {
+      const int owner = tok / per;
+      const float4 v = *reinterpret_cast<const float4*>(stg + (size_t)tok * TC_BLOCK_N + 4 * lane);
+      const uint32_t dst = dsmem_addr(smem_base + recv_off, (uint32_t)owner) +
+                           (uint32_t)((rank * per + (tok - owner * per)) * TC_BLOCK_N + 4 * lane) * 4u;
+      asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z),
+                   "f"(v.w)
+                   : "memory");
+    }
+    cluster_sync_all();                                        // every partial row has reached its owner
+  }
 
-  // ---------------- epilogue, part 2: owner-side reduction (local) + fused operation.
-  // A thread handles 4 consecutive features (quad = lane) of one row at a time; the four warps
-  // take rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 features
-  // (16 lanes) away, so they are exchanged with a warp shuffle.
-  if (warp >= 2) {
+  // ---------------- owner-side reduction + fused operation, all six warps.
+  // A thread handles 4 consecutive features (quad = lane) of one row at a time; the warps take
+  // rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 (or 32)
+  // features away, i.e. 16 (or 8) lanes, and are exchanged with a warp shuffle.
+  {
+    constexpr int RB = 6;                                      // rows per batch: their global loads fly together
+    constexpr int NW = TC_THREADS / 32;
     pdl_wait();
     const int t0 = rank * per, cnt = min(p.M, t0 + per) - t0;  // rows owned by this split
     const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
     const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
+    // per-row scale of unnormalised input rows (RMSNorm finished on the consumer side)
+    for (int i = threadIdx.x; i < cnt; i += TC_THREADS)
+      rstd_s[i] = p.in_sumsq ? rstd_from_sumsq(p.in_sumsq[t0 + i], p.norm_d, p.norm_eps) : 1.0f;
+    __syncthreads();
     float g4[4] = {1.f, 1.f, 1.f, 1.f};
     if (p.mode == EPI_RESID && n4 + 3 < p.N) {
       const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
@@ -404,85 +410,107 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
       const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
       g4[0] = a.x; g4[1] = a.y; g4[2] = b.x; g4[3] = b.y;
     }
-    for (int tl = warp - 2; tl < cnt; tl += 4) {
-      const int tok = t0 + tl;
-      float4 acc = *reinterpret_cast<const float4*>(red + (size_t)tl * TC_BLOCK_N + 4 * lane);
-      for (int r = 1; r < p.splits; ++r) {
-        const float4 v = *reinterpret_cast<const float4*>(red + (size_t)(r * per + tl) * TC_BLOCK_N + 4 * lane);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-      }
-      if (p.in_sumsq) {                                        // the input rows were left unnormalised
-        const float rs = rstd_from_sumsq(p.in_sumsq[tok], p.norm_d, p.norm_eps);
-        acc.x *= rs; acc.y *= rs; acc.z *= rs; acc.w *= rs;
-      }
-      if (p.mode == EPI_RESID) {
-        float ss = 0.f;
-        if (n4 + 3 < p.N) {                                    // N (the model width) is a multiple of 8
-          float4* xp = reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4);
-          float4 xv = *xp;
-          xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
-          *xp = xv;
-          uint2 pk;
-          pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
-          pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
-          *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
-          ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
-        }
-        ss = warp_sum(ss);
-        if (lane == 0) atomicAdd(p.out_sumsq + tok, sumsq_to_fixed(ss));
-      } else if (p.mode == EPI_STORE) {
-        float* dst = p.out + (size_t)tok * p.ldo + n4;
-        if (n4 + 3 < p.N && (p.ldo & 3) == 0) {
-          *reinterpret_cast<float4*>(dst) = acc;
-        } else {
-          if (n4 < p.N) dst[0] = acc.x;
-          if (n4 + 1 < p.N) dst[1] = acc.y;
-          if (n4 + 2 < p.N) dst[2] = acc.z;
-          if (n4 + 3 < p.N) dst[3] = acc.w;
-        }
-      } else if (p.mode == EPI_SWIGLU) {
-        // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
-        const float ux = __shfl_down_sync(0xffffffffu, acc.x, 16), uy = __shfl_down_sync(0xffffffffu, acc.y, 16);
-        const float uz = __shfl_down_sync(0xffffffffu, acc.z, 16), uw = __shfl_down_sync(0xffffffffu, acc.w, 16);
-        const int f = tile * 64 + 4 * lane;
-        if (lane < 16 && f < p.F) {                            // F is a multiple of 8: a quad is all in or all out
-          const float h0 = acc.x / (1.0f + __expf(-acc.x)) * ux, h1 = acc.y / (1.0f + __expf(-acc.y)) * uy;
-          const float h2 = acc.z / (1.0f + __expf(-acc.z)) * uz, h3 = acc.w / (1.0f + __expf(-acc.w)) * uw;
-          uint2 pk;
-          pk.x = pack_bf16x2(h0, h1);
-          pk.y = pack_bf16x2(h2, h3);
-          *reinterpret_cast<uint2*>(p.hf + (size_t)tok * p.F + f) = pk;
-        }
-      } else {                                                 // EPI_QKV
-        const int half = p.D >> 1;
-        const int sh = half >> 2;                              // partner quad is `sh` lanes away (16 or 8)
-        // partner values: the other half of the same head
-        const float wx = __shfl_xor_sync(0xffffffffu, acc.x, sh), wy = __shfl_xor_sync(0xffffffffu, acc.y, sh);
-        const float wz = __shfl_xor_sync(0xffffffffu, acc.z, sh), ww = __shfl_xor_sync(0xffffffffu, acc.w, sh);
-        if (n4 < p.N) {                                        // N is a multiple of D: a quad is all in or all out
-          const int head = n4 / p.D, dd = n4 - head * p.D;
-          const bool lo = dd < half;
-          const int j = lo ? dd : dd - half;
-          float4 r = acc;
-          if (head < p.H + p.H_kv) {
-            const float4 c01 = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + j);
-            const float4 c23 = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + j + 2);
-            const float sg = lo ? -1.f : 1.f;
-            r.x = acc.x * c01.x + sg * wx * c01.y;
-            r.y = acc.y * c01.z + sg * wy * c01.w;
-            r.z = acc.z * c23.x + sg * wz * c23.y;
-            r.w = acc.w * c23.z + sg * ww * c23.w;
+    // EPI_QKV: which head this quad belongs to
+    const int half = p.mode == EPI_QKV ? p.D >> 1 : 2;
+    const int sh = half >> 2;                                  // partner quad is `sh` lanes away (16 or 8)
+    const int head = p.mode == EPI_QKV ? n4 / p.D : 0, dd = p.mode == EPI_QKV ? n4 - head * p.D : 0;
+    const bool lo = dd < half;
+    const int jr = lo ? dd : dd - half;
+    const bool rot = p.mode == EPI_QKV && n4 < p.N && head < p.H + p.H_kv;
+    const bool in_n = n4 + 3 < p.N;
+    const float sg = lo ? -1.f : 1.f;
+
+    for (int tb = warp; tb < cnt; tb += NW * RB) {
+      float4 g0[RB], g1[RB];                                   // prefetched global operands of the batch
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        const int tl = tb + NW * u;
+        g0[u] = make_float4(1.f, 0.f, 1.f, 0.f);
+        g1[u] = make_float4(1.f, 0.f, 1.f, 0.f);
+        if (tl < cnt) {
+          const int tok = t0 + tl;
+          if (p.mode == EPI_RESID) {
+            if (in_n) g0[u] = *reinterpret_cast<const float4*>(p.x + (size_t)tok * p.N + n4);
+          } else if (rot) {
+            g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
+            g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
           }
-          uint2 pk;
-          pk.x = pack_bf16x2(r.x, r.y);
-          pk.y = pack_bf16x2(r.z, r.w);
-          const int slot = C + tok;
-          if (head < p.H) {
-            *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
-          } else if (slot < p.C_max) {
-            bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
-                                             : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
-            *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        const int tl = tb + NW * u;
+        if (tl >= cnt) break;                                  // warp-uniform
+        const int tok = t0 + tl;
+        float4 acc = *reinterpret_cast<const float4*>(recv + (size_t)tl * TC_BLOCK_N + 4 * lane);
+        for (int r = 1; r < p.splits; ++r) {
+          const float4 v = *reinterpret_cast<const float4*>(recv + (size_t)(r * per + tl) * TC_BLOCK_N + 4 * lane);
+          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const float rs = rstd_s[tl];
+        acc.x *= rs; acc.y *= rs; acc.z *= rs; acc.w *= rs;
+        if (p.mode == EPI_RESID) {
+          float ss = 0.f;
+          if (in_n) {                                          // N (the model width) is a multiple of 8
+            float4 xv = g0[u];
+            xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
+            *reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4) = xv;
+            uint2 pk;
+            pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
+            pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
+            *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
+            ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
+          }
+          ss = warp_sum(ss);
+          if (lane == 0) atomicAdd(p.out_sumsq + tok, sumsq_to_fixed(ss));
+        } else if (p.mode == EPI_STORE) {
+          float* dst = p.out + (size_t)tok * p.ldo + n4;
+          if (in_n && (p.ldo & 3) == 0) {
+            *reinterpret_cast<float4*>(dst) = acc;
+          } else {
+            if (n4 < p.N) dst[0] = acc.x;
+            if (n4 + 1 < p.N) dst[1] = acc.y;
+            if (n4 + 2 < p.N) dst[2] = acc.z;
+            if (n4 + 3 < p.N) dst[3] = acc.w;
+          }
+        } else if (p.mode == EPI_SWIGLU) {
+          // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
+          const float ux = __shfl_down_sync(0xffffffffu, acc.x, 16), uy = __shfl_down_sync(0xffffffffu, acc.y, 16);
+          const float uz = __shfl_down_sync(0xffffffffu, acc.z, 16), uw = __shfl_down_sync(0xffffffffu, acc.w, 16);
+          const int f = tile * 64 + 4 * lane;
+          if (lane < 16 && f < p.F) {                          // F is a multiple of 8: a quad is all in or all out
+            const float h0 = __fdividef(acc.x, 1.0f + __expf(-acc.x)) * ux;
+            const float h1 = __fdividef(acc.y, 1.0f + __expf(-acc.y)) * uy;
+            const float h2 = __fdividef(acc.z, 1.0f + __expf(-acc.z)) * uz;
+            const float h3 = __fdividef(acc.w, 1.0f + __expf(-acc.w)) * uw;
+            uint2 pk;
+            pk.x = pack_bf16x2(h0, h1);
+            pk.y = pack_bf16x2(h2, h3);
+            *reinterpret_cast<uint2*>(p.hf + (size_t)tok * p.F + f) = pk;
+          }
+        } else {                                               // EPI_QKV
+          // partner values: the other half of the same head
+          const float wx = __shfl_xor_sync(0xffffffffu, acc.x, sh), wy = __shfl_xor_sync(0xffffffffu, acc.y, sh);
+          const float wz = __shfl_xor_sync(0xffffffffu, acc.z, sh), ww = __shfl_xor_sync(0xffffffffu, acc.w, sh);
+          if (n4 < p.N) {                                      // N is a multiple of D: a quad is all in or all out
+            float4 r = acc;
+            if (rot) {
+              r.x = acc.x * g0[u].x + sg * wx * g0[u].y;
+              r.y = acc.y * g0[u].z + sg * wy * g0[u].w;
+              r.z = acc.z * g1[u].x + sg * wz * g1[u].y;
+              r.w = acc.w * g1[u].z + sg * ww * g1[u].w;
+            }
+            uint2 pk;
+            pk.x = pack_bf16x2(r.x, r.y);
+            pk.y = pack_bf16x2(r.z, r.w);
+            const int slot = C + tok;
+            if (head < p.H) {
+              *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
+            } else if (slot < p.C_max) {
+              bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
+                                               : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
+              *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
+            }
           }
         }
       }
