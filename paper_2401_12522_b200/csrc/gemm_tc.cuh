@@ -275,7 +275,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
 
   if (warp == 0) {
     // ---------------- TMA producer
-    if (lane == 0 && nkb > 0) {
+    if (nkb > 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       const int row_a = p.dual ? tile * 64 : tile * TC_BLOCK_N;
       auto load_a = [&](int i) {
@@ -296,23 +296,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         tma_load_2d(smem_base + (uint32_t)s * stage_bytes + a_bytes, &map_b, (kb0 + i) * TC_BLOCK_K, 0,
                     smem_u32(&bar_full[s]), pol_x);
       };
-      // weights do not depend on earlier kernels: fill the ring with them first, then wait for
-      // the producer of the activations
+      // Weights do not depend on earlier kernels: the first ring fill requests them before the
+      // kernel waits for the producer of the activations.  One lane per stage issues that first
+      // fill, so the requests leave together; lane 0 alone runs the steady state.
       const int npre = nkb < p.stages ? nkb : p.stages;
-      for (int i = 0; i < npre; ++i) load_a(i);
+      if (lane < npre) load_a(lane);
       pdl_wait();
-      for (int i = 0; i < npre; ++i) load_b(i);
-      bool ok = true;
-      for (int i = npre; i < nkb; ++i) {
-        const int s = i % p.stages;
-        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, p.status);
-        if (!ok) break;
-        load_a(i);
-        load_b(i);
-      }
-      if (!ok) {
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);      // let the copies in flight land
+      if (lane < npre) load_b(lane);
+      __syncwarp();
+      if (lane == 0) {
+        bool ok = true;
+        for (int i = npre; i < nkb; ++i) {
+          const int s = i % p.stages;
+          const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+          ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, p.status);
+          if (!ok) break;
+          load_a(i);
+          load_b(i);
+        }
+        if (!ok) {
+          for (int i = 0; i < 64; ++i) __nanosleep(1000);    // let the copies in flight land
+        }
       }
     }
   } else if (warp == 1) {
@@ -421,88 +425,131 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     const float sg = lo ? -1.f : 1.f;
 
     for (int tb = warp; tb < cnt; tb += NW * RB) {
-      float4 g0[RB], g1[RB];                                   // prefetched global operands of the batch
+      // phase A: every load of the batch (global operands, partial sums, row scales)
+      float4 g0[RB], g1[RB], acc[RB];
+      float rs[RB];
+      bool live[RB];
 #pragma unroll
       for (int u = 0; u < RB; ++u) {
         const int tl = tb + NW * u;
+        live[u] = tl < cnt;
+        const int tlc = live[u] ? tl : tb;                     // clamp: dead rows recompute row tb, store nothing
+        const int tok = t0 + tlc;
         g0[u] = make_float4(1.f, 0.f, 1.f, 0.f);
         g1[u] = make_float4(1.f, 0.f, 1.f, 0.f);
-        if (tl < cnt) {
-          const int tok = t0 + tl;
-          if (p.mode == EPI_RESID) {
-            if (in_n) g0[u] = *reinterpret_cast<const float4*>(p.x + (size_t)tok * p.N + n4);
-          } else if (rot) {
-            g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
-            g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
-          }
+        if (p.mode == EPI_RESID) {
+          if (in_n) g0[u] = *reinterpret_cast<const float4*>(p.x + (size_t)tok * p.N + n4);
+        } else if (rot) {
+          g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
+          g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
+        }
+        acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
+        rs[u] = rstd_s[tlc];
+      }
+      for (int r = 1; r < p.splits; ++r) {                     // split order: fixed summation order
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          const int tlc = live[u] ? tb + NW * u : tb;
+          const float4 v = *reinterpret_cast<const float4*>(recv + (size_t)(r * per + tlc) * TC_BLOCK_N + 4 * lane);
+          acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
         }
       }
 #pragma unroll
-      for (int u = 0; u < RB; ++u) {
-        const int tl = tb + NW * u;
-        if (tl >= cnt) break;                                  // warp-uniform
-        const int tok = t0 + tl;
-        float4 acc = *reinterpret_cast<const float4*>(recv + (size_t)tl * TC_BLOCK_N + 4 * lane);
-        for (int r = 1; r < p.splits; ++r) {
-          const float4 v = *reinterpret_cast<const float4*>(recv + (size_t)(r * per + tl) * TC_BLOCK_N + 4 * lane);
-          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        const float rs = rstd_s[tl];
-        acc.x *= rs; acc.y *= rs; acc.z *= rs; acc.w *= rs;
-        if (p.mode == EPI_RESID) {
-          float ss = 0.f;
+      for (int u = 0; u < RB; ++u) { acc[u].x *= rs[u]; acc[u].y *= rs[u]; acc[u].z *= rs[u]; acc[u].w *= rs[u]; }
+
+      // phase B: the fused operation, written batch-wide so that independent rows interleave
+      if (p.mode == EPI_RESID) {
+        float ss[RB];
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          ss[u] = 0.f;
           if (in_n) {                                          // N (the model width) is a multiple of 8
             float4 xv = g0[u];
-            xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
-            *reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4) = xv;
-            uint2 pk;
-            pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
-            pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
-            *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
-            ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
+            xv.x += acc[u].x; xv.y += acc[u].y; xv.z += acc[u].z; xv.w += acc[u].w;
+            ss[u] = live[u] ? xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w : 0.f;
+            if (live[u]) {
+              const int tok = t0 + tb + NW * u;
+              *reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4) = xv;
+              uint2 pk;
+              pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
+              pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
+              *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
+            }
           }
-          ss = warp_sum(ss);
-          if (lane == 0) atomicAdd(p.out_sumsq + tok, sumsq_to_fixed(ss));
-        } else if (p.mode == EPI_STORE) {
-          float* dst = p.out + (size_t)tok * p.ldo + n4;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int u = 0; u < RB; ++u) ss[u] += __shfl_xor_sync(0xffffffffu, ss[u], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+          for (int u = 0; u < RB; ++u)
+            if (live[u]) atomicAdd(p.out_sumsq + t0 + tb + NW * u, sumsq_to_fixed(ss[u]));
+        }
+      } else if (p.mode == EPI_STORE) {
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          if (!live[u]) continue;
+          float* dst = p.out + (size_t)(t0 + tb + NW * u) * p.ldo + n4;
           if (in_n && (p.ldo & 3) == 0) {
-            *reinterpret_cast<float4*>(dst) = acc;
+            *reinterpret_cast<float4*>(dst) = acc[u];
           } else {
-            if (n4 < p.N) dst[0] = acc.x;
-            if (n4 + 1 < p.N) dst[1] = acc.y;
-            if (n4 + 2 < p.N) dst[2] = acc.z;
-            if (n4 + 3 < p.N) dst[3] = acc.w;
+            if (n4 < p.N) dst[0] = acc[u].x;
+            if (n4 + 1 < p.N) dst[1] = acc[u].y;
+            if (n4 + 2 < p.N) dst[2] = acc[u].z;
+            if (n4 + 3 < p.N) dst[3] = acc[u].w;
           }
-        } else if (p.mode == EPI_SWIGLU) {
-          // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
-          const float ux = __shfl_down_sync(0xffffffffu, acc.x, 16), uy = __shfl_down_sync(0xffffffffu, acc.y, 16);
-          const float uz = __shfl_down_sync(0xffffffffu, acc.z, 16), uw = __shfl_down_sync(0xffffffffu, acc.w, 16);
-          const int f = tile * 64 + 4 * lane;
-          if (lane < 16 && f < p.F) {                          // F is a multiple of 8: a quad is all in or all out
-            const float h0 = __fdividef(acc.x, 1.0f + __expf(-acc.x)) * ux;
-            const float h1 = __fdividef(acc.y, 1.0f + __expf(-acc.y)) * uy;
-            const float h2 = __fdividef(acc.z, 1.0f + __expf(-acc.z)) * uz;
-            const float h3 = __fdividef(acc.w, 1.0f + __expf(-acc.w)) * uw;
+        }
+      } else if (p.mode == EPI_SWIGLU) {
+        // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
+        float4 up[RB];
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          up[u].x = __shfl_down_sync(0xffffffffu, acc[u].x, 16);
+          up[u].y = __shfl_down_sync(0xffffffffu, acc[u].y, 16);
+          up[u].z = __shfl_down_sync(0xffffffffu, acc[u].z, 16);
+          up[u].w = __shfl_down_sync(0xffffffffu, acc[u].w, 16);
+        }
+        const int f = tile * 64 + 4 * lane;
+        if (lane < 16 && f < p.F) {                            // F is a multiple of 8: a quad is all in or all out
+#pragma unroll
+          for (int u = 0; u < RB; ++u) {
+            const float h0 = __fdividef(acc[u].x, 1.0f + __expf(-acc[u].x)) * up[u].x;
+            const float h1 = __fdividef(acc[u].y, 1.0f + __expf(-acc[u].y)) * up[u].y;
+            const float h2 = __fdividef(acc[u].z, 1.0f + __expf(-acc[u].z)) * up[u].z;
+            const float h3 = __fdividef(acc[u].w, 1.0f + __expf(-acc[u].w)) * up[u].w;
             uint2 pk;
             pk.x = pack_bf16x2(h0, h1);
             pk.y = pack_bf16x2(h2, h3);
-            *reinterpret_cast<uint2*>(p.hf + (size_t)tok * p.F + f) = pk;
+            if (live[u]) *reinterpret_cast<uint2*>(p.hf + (size_t)(t0 + tb + NW * u) * p.F + f) = pk;
           }
-        } else {                                               // EPI_QKV
-          // partner values: the other half of the same head
-          const float wx = __shfl_xor_sync(0xffffffffu, acc.x, sh), wy = __shfl_xor_sync(0xffffffffu, acc.y, sh);
-          const float wz = __shfl_xor_sync(0xffffffffu, acc.z, sh), ww = __shfl_xor_sync(0xffffffffu, acc.w, sh);
-          if (n4 < p.N) {                                      // N is a multiple of D: a quad is all in or all out
-            float4 r = acc;
+        }
+      } else {                                                 // EPI_QKV
+        // partner values: the other half of the same head
+        float4 w[RB];
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          w[u].x = __shfl_xor_sync(0xffffffffu, acc[u].x, sh);
+          w[u].y = __shfl_xor_sync(0xffffffffu, acc[u].y, sh);
+          w[u].z = __shfl_xor_sync(0xffffffffu, acc[u].z, sh);
+          w[u].w = __shfl_xor_sync(0xffffffffu, acc[u].w, sh);
+        }
+        if (n4 < p.N) {                                        // N is a multiple of D: a quad is all in or all out
+#pragma unroll
+          for (int u = 0; u < RB; ++u) {
+            float4 r = acc[u];
             if (rot) {
-              r.x = acc.x * g0[u].x + sg * wx * g0[u].y;
-              r.y = acc.y * g0[u].z + sg * wy * g0[u].w;
-              r.z = acc.z * g1[u].x + sg * wz * g1[u].y;
-              r.w = acc.w * g1[u].z + sg * ww * g1[u].w;
+              r.x = acc[u].x * g0[u].x + sg * w[u].x * g0[u].y;
+              r.y = acc[u].y * g0[u].z + sg * w[u].y * g0[u].w;
+              r.z = acc[u].z * g1[u].x + sg * w[u].z * g1[u].y;
+              r.w = acc[u].w * g1[u].z + sg * w[u].w * g1[u].w;
             }
             uint2 pk;
             pk.x = pack_bf16x2(r.x, r.y);
             pk.y = pack_bf16x2(r.z, r.w);
+            if (!live[u]) continue;
+            const int tok = t0 + tb + NW * u;
             const int slot = C + tok;
             if (head < p.H) {
               *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
