@@ -361,7 +361,7 @@ void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
   if (w > 8) w = 8;
   const int rt = (M + 16 * w - 1) / (16 * w);
   const int ctas = H * B * rt;
-  int s = (296 + ctas - 1) / ctas;
+  int s = 296 / ctas;                          // every slice resident at once (two CTAs per SM)
   if (s < 1) s = 1;
   if (s > 6) s = 6;
   *warps = w; *row_tiles = rt; *splits = s;
