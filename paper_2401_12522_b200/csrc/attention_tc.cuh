@@ -74,8 +74,10 @@ __device__ __forceinline__ uint32_t swz(int r, int c) {
   return (uint32_t)(r * (D * 2) + ((c ^ (r & 7)) << 4));
 }
 
-template <int D>
-__global__ void __launch_bounds__(256) k_attn_tc(AttnArgs a) {
+// MAXW = most warps a CTA of this instantiation is launched with: blocks of up to 5 warps (80 query
+// rows, the 69-row step block) are compiled to fit two per SM.
+template <int D, int MAXW>
+__global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnArgs a) {
   constexpr int CH = D / 8;                  // 16-byte chunks per row
   constexpr int NT_S = ATT_KEYS / 8;         // score n-tiles per chunk
   constexpr int NT_O = D / 8;                // output n-tiles

@@ -361,7 +361,8 @@ void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
   if (w > 8) w = 8;
   const int rt = (M + 16 * w - 1) / (16 * w);
   const int ctas = H * B * rt;
-  int s = 296 / ctas;                          // every slice resident at once (two CTAs per SM)
+  static const int target = getenv("BITA_ATTN_CTAS") ? atoi(getenv("BITA_ATTN_CTAS")) : 296;
+  int s = target / ctas;                       // every slice resident at once (two CTAs per SM)
   if (s < 1) s = 1;
   if (s > 6) s = 6;
   *warps = w; *row_tiles = rt; *splits = s;
@@ -498,17 +499,24 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s) {
                       rows_cta + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
     attr_set = true;
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
+  const dim3 blk(a.warps * 32);
   int rc;
   if (a.D == 128) {
-    if ((rc = launch(s, pdl, g1, dim3(a.warps * 32), smem, 1, k_attn_tc<128>, a))) return rc;
+    rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 5>, a)
+                      : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 8>, a);
+    if (rc) return rc;
     return launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a);
   }
-  if ((rc = launch(s, pdl, g1, dim3(a.warps * 32), smem, 1, k_attn_tc<64>, a))) return rc;
+  rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 5>, a)
+                    : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 8>, a);
+  if (rc) return rc;
   return launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
 
