@@ -259,46 +259,20 @@ struct GemmDesc {
   size_t bytes = 0;                        // bytes of each
 };
 
-// Split-K factor (= cluster size).  A kernel launched as clusters gets one CTA per SM and a
-// cluster-size-dependent number of clusters at a time (the runtime reports it), so a split is only
-// worth it when all its CTAs run in one wave; tile counts above the SM count run unsplit with two
-// CTAs per SM.
-int max_active_clusters(int cluster) {
-  static int cache[9] = {0};
-  if (cluster < 1 || cluster > 8) return 0;
-  if (!cache[cluster]) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(cluster * 32, cluster);
-    cfg.blockDim = dim3(TC_THREADS);
-    cfg.dynamicSmemBytes = 200 * 1024;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 1;
-    at[0].val.clusterDim.y = cluster;
-    at[0].val.clusterDim.z = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = 1;
-    int n = 0;
-    cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-    if (cudaOccupancyMaxActiveClusters(&n, k_gemm_tc, &cfg) != cudaSuccess || n < 1) {
-      static const int fallback[9] = {0, 148, 74, 45, 33, 26, 22, 18, 15};   // what a B200 reported
-      n = fallback[cluster];
-      cudaGetLastError();
-    }
-    cache[cluster] = n;
-  }
-  return cache[cluster];
-}
+// Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
+// shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
+constexpr int GEMM_MAX_CTAS = 296;
+constexpr int GEMM_MAX_SPLITS = 4;
 
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  static const int cap = getenv("BITA_SPLIT_CAP") ? atoi(getenv("BITA_SPLIT_CAP")) : 8;
-  int best = 1;
-  for (int s = 2; s <= 8 && s <= max_splits && s <= cap; ++s) {
-    if (kb / s < 4) break;
-    if (tiles <= max_active_clusters(s)) best = s;            // all tiles * s CTAs resident at once
-  }
-  return best;
+  static const int cap = getenv("BITA_SPLIT_CAP") ? atoi(getenv("BITA_SPLIT_CAP")) : GEMM_MAX_SPLITS;
+  int s = GEMM_MAX_CTAS / tiles;
+  if (s > kb / 4) s = kb / 4;
+  if (s > max_splits) s = max_splits;
+  if (s > cap) s = cap;
+  if (s < 1) s = 1;
+  return s;
 }
 
 int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
@@ -337,20 +311,19 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
   const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  // One wave with one CTA per SM gets the whole shared memory; more tiles than SMs share it two per SM.
-  const bool two_per_sm = splits == 1 && g.tiles > 148 && n_pad <= 96;
+  // Small blocks run two CTAs per SM (half the shared memory each); large ones one per SM, and
+  // then a split only pays while all its CTAs fit in one wave.
+  const bool two_per_sm = n_pad <= 96;
+  if (!two_per_sm && g.tiles * splits > 148) splits = 148 / g.tiles > 0 ? 148 / g.tiles : 1;
   const size_t budget = (two_per_sm ? 110 : 220) * 1024;
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
-  // the epilogue reuses the stages for its staging and receive buffers
-  if ((size_t)stages * stage < ((size_t)2 * M + splits) * TC_BLOCK_N * 4) splits = 1;
-  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;
+  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // staging of a whole tile
   p.splits = splits;
   p.stages = stages;
   const size_t smem = stages * stage + 1024;
-  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, (unsigned)splits, k_gemm_tc, g.a0, g.a1,
-                map_b, p);
+  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc, g.a0, g.a1, map_b, p);
 }
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
@@ -377,7 +350,7 @@ int attn_splits(int H, int B, int M) {
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
-  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc;
+  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
 };
@@ -406,6 +379,8 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   const size_t S = 6;                        // upper bound of attn_splits
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
+  t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
+  t.gemm_cnt = (int32_t*)take(4096 * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -478,6 +453,8 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
     it = c->act_maps.emplace(key, m).first;
   }
   p.status = &c->b.state->status;
+  p.part = c->b.gemm_part;
+  p.tile_counters = c->b.gemm_cnt;
   Timed t(c, 0);
   int rc = launch_gemm_tc(g, it->second, n_pad, M, p, c->pdl, c->stream);
   c->launches++;
@@ -694,6 +671,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   }
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
+  if (cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
@@ -852,9 +830,12 @@ const char* bita_strerror(int code) {
 
 int bita_last_cuda_error(void) { return g_last_cuda_error; }
 
+// Workspace of the stand-alone projection: status word, tile counters, split-K exchange buffer.
 int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes) {
   if (!out_bytes || M < 1 || M > BITA_MAX_ROWS || N < 1 || K < 8 || K % 8) return BITA_ERR_INVALID_ARG;
-  *out_bytes = ALIGN;                                         // one status word
+  const int tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
+  const int splits = gemm_splits(tiles, K, 8);
+  *out_bytes = ALIGN + align_up((size_t)tiles * 4) + align_up(splits > 1 ? (size_t)tiles * splits * M * TC_BLOCK_N * 4 : 0);
   return BITA_OK;
 }
 
@@ -871,9 +852,12 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   const int n_pad = pad16(M);
   CUtensorMap mb;
   if ((rc = make_map(&mb, X, K, M, n_pad))) return rc;
-  CU_TRY(cudaMemsetAsync(workspace, 0, 4, s));
+  const size_t cnt_bytes = align_up((size_t)g.tiles * 4);
+  CU_TRY(cudaMemsetAsync(workspace, 0, ALIGN + cnt_bytes, s));     // status word and tile counters start at zero
   GemmTcParams p = epi_store((float*)Y, N);
   p.status = (int32_t*)workspace;
+  p.tile_counters = (int32_t*)((uint8_t*)workspace + ALIGN);
+  p.part = (float*)((uint8_t*)workspace + ALIGN + cnt_bytes);
   if ((rc = launch_gemm_tc(g, mb, n_pad, M, p, false, s))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;

@@ -8,12 +8,12 @@
 // columns).  Each CTA owns one tile of 128 output features and a contiguous range of 64-wide K
 // blocks (split-K); it streams its weight tiles through a ring of TMA-filled, 128-byte-swizzled
 // shared-memory stages, one elected thread issues tcgen05.mma into a TMEM accumulator, and four
-// epilogue warps read the accumulator back with tcgen05.ld.  The splits of one tile form a
-// thread-block cluster: each split owns a slice of the block's rows, every split sends its partial
-// values for a row to the owner's shared memory (distributed shared memory stores), and after one
-// cluster barrier each owner sums its rows over the splits, always in split order - every output
-// is a fixed-order sum (deterministic, and independent of how many other rows the block holds)
-// and no partial result ever goes to HBM.  The owner then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
+// epilogue warps read the accumulator back with tcgen05.ld.  With split-K every split stores its
+// partial tile in an L2-resident exchange buffer and bumps a per-tile counter; the split that
+// completes the counter sums the partial tiles, always in split order - every output is a
+// fixed-order sum (deterministic, and independent of how many other rows the block holds), no CTA
+// waits for another, and the splits that are not last leave at once, which frees their SM for the
+// next kernel's prologue.  The reducing CTA then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
 // builds the 128-row weight tile from 64 gate rows and the 64 matching up rows, so both halves of
 // a product sit in the same tile); or rotary embedding with the q rows going to a bf16 buffer and
 // the k/v rows straight into the KV cache.
@@ -65,11 +65,13 @@ struct GemmTcParams {
   int32_t K;
   int32_t n_pad;         // MMA N: rows of X padded to a multiple of 16
   int32_t stages;
-  int32_t splits;        // = cluster size along y; split s of a tile is cluster rank s
+  int32_t splits;        // split-K factor = gridDim.y
   int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1
   int32_t tmem_cols;     // power of two >= max(32, n_pad)
   int32_t mode;          // GemmEpilogue
   int32_t* status;       // device status word (sticky error flag)
+  float* part;           // split-K exchange buffer [tiles][splits][M][128] fp32 (splits > 1)
+  int32_t* tile_counters;  // [tiles], zero before the launch; left zero by the kernel
   // row scale of the input (RMSNorm statistics of the rows of X), or null: y *= rstd(row)
   const unsigned long long* in_sumsq;
   int32_t norm_d;
@@ -204,28 +206,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// Thread-block cluster helpers (split-K partners form one cluster).
-__device__ __forceinline__ uint32_t cluster_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
-}
-// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void dsmem_st(uint32_t addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
           const __grid_constant__ CUtensorMap map_b, GemmTcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -234,6 +216,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t bar_acc;
   __shared__ uint32_t tmem_base_slot;
   __shared__ float rstd_s[BITA_MAX_ROWS];
+  __shared__ int last_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -343,25 +326,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
   }
 
-  // ---------------- epilogue
-  // The pipeline stages are free once the accumulator barrier has completed; they are reused as
-  //   stg  [M][128] fp32           this split's partial tile, row-major
-  //   recv [splits][per][128] fp32 (splits > 1) partial values of the rows this split owns
-  // Split r of the cluster owns rows [r * per, (r + 1) * per).  Part 1 moves the accumulator to
-  // `stg` (thread = feature).  With splits > 1 every split then sends each row of `stg` to the
-  // row's owner as 16-byte distributed-shared-memory stores, and after one cluster barrier the
-  // owner sums its rows over the source splits, in split order, from local memory.
+  // ---------------- epilogue, part 1: accumulator -> staging
+  // splits == 1: the tile goes to shared memory (`stg`, the pipeline stages, free once the
+  //              accumulator barrier has completed), row-major [M][128] fp32.
+  // splits  > 1: every split stores its partial tile to the global exchange buffer
+  //              part[tile][split][M][128] (L2-resident, overwritten by every projection), then
+  //              bumps the tile's counter; the split that finds the counter complete sums the
+  //              partial tiles, always in split order, and applies the fused operation.  No CTA
+  //              ever waits for another, and the early leavers free their SM for the next kernel.
   float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
-  const int per = (p.M + p.splits - 1) / p.splits;             // rows per owner
-  const int rank = p.splits > 1 ? (int)cluster_rank() : 0;
-  const uint32_t recv_off = (uint32_t)p.M * TC_BLOCK_N * 4u;   // byte offset of `recv` from the buffer base
-  const float* recv = p.splits > 1 ? stg + (size_t)p.M * TC_BLOCK_N : stg;
+  const size_t tile_elems = (size_t)p.M * TC_BLOCK_N;
+  float* part_tile = p.part + (size_t)tile * p.splits * tile_elems;      // this tile's partials, split-major
   if (warp >= 2) {
     const int lg = warp & 3;                                   // TMEM lane group this warp may read
     const int fr = lg * 32 + lane;                             // feature row of the tile owned by this thread
     bool ok = true;
     if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     tc_fence_after();
+    // the exchange buffer was last read by an earlier projection: be sure that one has finished
+    if (p.splits > 1) pdl_wait();
+    float* dst = p.splits > 1 ? part_tile + (size_t)split * tile_elems : stg;
     for (int c = 0; c < p.n_pad; c += 16) {
       float v[16];
       if (nkb > 0 && ok) {
@@ -372,31 +356,32 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
       }
 #pragma unroll
       for (int j = 0; j < 16; ++j)
-        if (c + j < p.M) stg[(c + j) * TC_BLOCK_N + fr] = v[j];
+        if (c + j < p.M) dst[(c + j) * TC_BLOCK_N + fr] = v[j];
     }
+    if (p.splits > 1) __threadfence();
   }
   tc_fence_before();
   __syncthreads();
+  bool reducer = true;
   if (p.splits > 1) {
-    // a partner may only write into this CTA's stages once this CTA's own pipeline has drained
-    cluster_sync_all();
-    for (int tok = warp; tok < p.M; tok += TC_THREADS / 32) {
-      const int owner = tok / per;
-      const float4 v = *reinterpret_cast<const float4*>(stg + (size_t)tok * TC_BLOCK_N + 4 * lane);
-      const uint32_t dst = dsmem_addr(smem_base + recv_off, (uint32_t)owner) +
-                           (uint32_t)((rank * per + (tok - owner * per)) * TC_BLOCK_N + 4 * lane) * 4u;
-      asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z),
-                   "f"(v.w)
-                   : "memory");
+    if (threadIdx.x == 0) {
+      const int old = atomicAdd(p.tile_counters + tile, 1);
+      last_flag = old == p.splits - 1;
+      if (last_flag) p.tile_counters[tile] = 0;                // ready for the next projection
     }
-    cluster_sync_all();                                        // every partial row has reached its owner
+    __syncthreads();
+    reducer = last_flag != 0;
+    if (reducer) __threadfence();
   }
+  const float* recv = p.splits > 1 ? part_tile : stg;
+  const int per = p.M;                                         // row stride between the splits' partial tiles
+  const int rank = 0;
 
-  // ---------------- owner-side reduction + fused operation, all six warps.
+  // ---------------- epilogue, part 2: reduction over the splits + fused operation, all six warps.
   // A thread handles 4 consecutive features (quad = lane) of one row at a time; the warps take
   // rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 (or 32)
   // features away, i.e. 16 (or 8) lanes, and are exchanged with a warp shuffle.
-  {
+  if (reducer) {
     constexpr int RB = 6;                                      // rows per batch: their global loads fly together
     constexpr int NW = TC_THREADS / 32;
     pdl_wait();
@@ -443,14 +428,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
           g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
           g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
         }
-        acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
+        acc[u] = p.splits > 1 ? __ldcg(reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane))
+                              : *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
         rs[u] = rstd_s[tlc];
       }
       for (int r = 1; r < p.splits; ++r) {                     // split order: fixed summation order
 #pragma unroll
         for (int u = 0; u < RB; ++u) {
           const int tlc = live[u] ? tb + NW * u : tb;
-          const float4 v = *reinterpret_cast<const float4*>(recv + (size_t)(r * per + tlc) * TC_BLOCK_N + 4 * lane);
+          const float4 v = __ldcg(reinterpret_cast<const float4*>(recv + (size_t)(r * per + tlc) * TC_BLOCK_N + 4 * lane));
           acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
         }
       }
