@@ -562,8 +562,18 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   }
   if (want_logits) {
     if ((rc = gemm(c, c->d_head, b.xn, M, with_norm(epi_store(b.logits, m.V), 2 * m.L)))) return rc;
-    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select, P, (const float*)b.logits, m.V, b.sel_id, b.sel_val)))
-      return rc;
+    {
+      const size_t row_bytes = (size_t)m.V * 4;
+      const int use_smem = row_bytes <= 200 * 1024 ? 1 : 0;
+      static bool sel_attr = false;
+      if (!sel_attr) {
+        CU_TRY(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        sel_attr = true;
+      }
+      if ((rc = launch(s, pdl, dim3(M), dim3(1024), use_smem ? row_bytes : 0, 1, k_select, P, (const float*)b.logits,
+                       m.V, use_smem, b.sel_id, b.sel_val)))
+        return rc;
+    }
     c->launches += 1;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,

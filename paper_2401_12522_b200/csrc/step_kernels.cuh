@@ -73,10 +73,11 @@ __device__ __forceinline__ bool before(float v1, int i1, float v2, int i2) {
   return v1 > v2 || (v1 == v2 && i1 < i2);
 }
 
-__global__ void k_select(DevPlan plan, const float* __restrict__ logits, int V, int32_t* __restrict__ sel_id,
-                         float* __restrict__ sel_val) {
+__global__ void __launch_bounds__(1024) k_select(DevPlan plan, const float* __restrict__ logits, int V, int use_smem,
+                                                 int32_t* __restrict__ sel_id, float* __restrict__ sel_val) {
   pdl_launch();
   pdl_wait();
+  extern __shared__ float srow[];            // the row, kept on chip for the later passes (when it fits)
   __shared__ float sv[32];
   __shared__ int si[32];
   __shared__ float pv;
@@ -90,11 +91,28 @@ __global__ void k_select(DevPlan plan, const float* __restrict__ logits, int V, 
   for (int t = 0; t < K; ++t) {
     float bv = -INFINITY;
     int bi = 0x7fffffff;
-    for (int c = threadIdx.x; c < V; c += blockDim.x) {
-      const float v = row[c];
-      if (!(v == v)) continue;
-      if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;  // not strictly after the previous pick
-      if (before(v, c, bv, bi)) { bv = v; bi = c; }
+    if (t == 0 && (V & 3) == 0) {
+      // first pass: 16-byte loads from global memory, copy to shared memory on the way
+      const float4* row4 = reinterpret_cast<const float4*>(row);
+      for (int c4 = threadIdx.x; c4 < (V >> 2); c4 += blockDim.x) {
+        const float4 q = row4[c4];
+        if (use_smem && K > 1) reinterpret_cast<float4*>(srow)[c4] = q;
+        const float vals[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float v = vals[e];
+          const int c = 4 * c4 + e;
+          if (v == v && before(v, c, bv, bi)) { bv = v; bi = c; }
+        }
+      }
+    } else {
+      const float* src = (t > 0 && use_smem && (V & 3) == 0) ? srow : row;
+      for (int c = threadIdx.x; c < V; c += blockDim.x) {
+        const float v = src[c];
+        if (!(v == v)) continue;
+        if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;  // not strictly after the previous pick
+        if (before(v, c, bv, bi)) { bv = v; bi = c; }
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
