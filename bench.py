@@ -220,6 +220,22 @@ def ctx_len(ctx):
     return ctx._len
 
 
+def replica_plan(rank: int, shape):
+    """What differs between the independent replicas of a multi-GPU run: only the prompt seed."""
+    return {"prompt_seed": PROMPT_SEED + rank, "model_seed": MODEL_SEED, "plant_seed": PLANT_SEED}
+
+
+def aggregate_over_ranks(dist_mod, world: int, dev_ms: float, e2e_ms: float, tokens: float, device):
+    """Whole-job numbers of a replica run: the slowest rank's times, the sum of the tokens."""
+    times = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=device)
+    toks = torch.tensor([float(tokens)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist_mod.all_reduce(times, op=dist_mod.ReduceOp.MAX)
+        dist_mod.all_reduce(toks, op=dist_mod.ReduceOp.SUM)
+    dev_ms, e2e_ms = times.tolist()
+    return dev_ms, e2e_ms, float(toks[0])
+
+
 def run_ours(args, shape, tmpl):
     from paper_2401_12522_b200 import Bita
     from paper_2401_12522_b200.build import build
@@ -242,7 +258,7 @@ def run_ours(args, shape, tmpl):
     C_max = shape.prompt_len + total_steps * (depth + 1) + depth + rows + 64
     # replicas: every rank decodes its own sequence with its own seeds; no data-path collective
     weights = synth.make_weights(shape, MODEL_SEED, dtype=torch.bfloat16, device=dev)
-    prompt = synth.uniform_ints(PROMPT_SEED + rank, 5001, shape.prompt_len, shape.V).tolist()
+    prompt = synth.uniform_ints(replica_plan(rank, shape)["prompt_seed"], 5001, shape.prompt_len, shape.V).tolist()
     ctx = Bita(shape, weights, tmpl, C_max=C_max, device=dev)
 
     def start():
@@ -307,13 +323,8 @@ def run_ours(args, shape, tmpl):
     ctx.set_kernel_timing(False)
     ctx.step_finish()
 
-    times = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
-    toks = torch.tensor([float(tokens_timed)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    dev_ms, e2e_ms = times.tolist()
-    total_tokens = float(toks[0])
+    dev_ms, e2e_ms, total_tokens = aggregate_over_ranks(dist if world > 1 else None, world, dev_ms, e2e_ms,
+                                                        tokens_timed, dev)
 
     if rank == 0:
         peak, peak_src = _peaks()
@@ -354,7 +365,7 @@ def run_ours(args, shape, tmpl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(synth.CONFIGS))
