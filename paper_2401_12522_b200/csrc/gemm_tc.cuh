@@ -340,11 +340,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   if (warp >= 2) {
     const int lg = warp & 3;                                   // TMEM lane group this warp may read
     const int fr = lg * 32 + lane;                             // feature row of the tile owned by this thread
+    // While the main loop streams: wait for the earlier kernels (their outputs are read below, and
+    // the exchange buffer was last read by an earlier projection) and fetch the per-row scales of
+    // the unnormalised input rows (RMSNorm finished on the consumer side).
+    pdl_wait();
+    for (int i = threadIdx.x - 64; i < p.M; i += 128)
+      rstd_s[i] = p.in_sumsq ? rstd_from_sumsq(p.in_sumsq[i], p.norm_d, p.norm_eps) : 1.0f;
     bool ok = true;
     if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status);
     tc_fence_after();
-    // the exchange buffer was last read by an earlier projection: be sure that one has finished
-    if (p.splits > 1) pdl_wait();
     float* dst = p.splits > 1 ? part_tile + (size_t)split * tile_elems : stg;
     for (int c = 0; c < p.n_pad; c += 16) {
       float v[16];
@@ -371,10 +375,41 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
     __syncthreads();
     reducer = last_flag != 0;
-    if (reducer) __threadfence();
+    if (reducer) {
+      __threadfence();
+      // Sum the partial tiles into `stg`, in split order.  Each thread takes 16-byte items of the
+      // tile; the loads of four items (all their splits) are in flight together.
+      const int items = p.M * (TC_BLOCK_N / 4);
+      const float4* src = reinterpret_cast<const float4*>(part_tile);
+      const int stride4 = (int)(tile_elems / 4);               // between the splits' tiles
+      for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
+        float4 v[4][4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = min(i0 + u * TC_THREADS, items - 1);
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+            if (r < p.splits) v[u][r] = __ldcg(src + (size_t)r * stride4 + i);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * TC_THREADS;
+          float4 a4 = v[u][0];
+#pragma unroll
+          for (int r = 1; r < 4; ++r)
+            if (r < p.splits) { a4.x += v[u][r].x; a4.y += v[u][r].y; a4.z += v[u][r].z; a4.w += v[u][r].w; }
+          for (int r = 4; r < p.splits; ++r) {                 // more than four splits: the rest one by one
+            const float4 w = __ldcg(src + (size_t)r * stride4 + min(i, items - 1));
+            a4.x += w.x; a4.y += w.y; a4.z += w.z; a4.w += w.w;
+          }
+          if (i < items) reinterpret_cast<float4*>(stg)[i] = a4;
+        }
+      }
+      __syncthreads();
+    }
   }
-  const float* recv = p.splits > 1 ? part_tile : stg;
-  const int per = p.M;                                         // row stride between the splits' partial tiles
+  const float* recv = stg;
+  const int per = p.M;
   const int rank = 0;
 
   // ---------------- epilogue, part 2: reduction over the splits + fused operation, all six warps.
@@ -388,10 +423,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     const int t0 = rank * per, cnt = min(p.M, t0 + per) - t0;  // rows owned by this split
     const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
     const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
-    // per-row scale of unnormalised input rows (RMSNorm finished on the consumer side)
-    for (int i = threadIdx.x; i < cnt; i += TC_THREADS)
-      rstd_s[i] = p.in_sumsq ? rstd_from_sumsq(p.in_sumsq[t0 + i], p.norm_d, p.norm_eps) : 1.0f;
-    __syncthreads();
     float g4[4] = {1.f, 1.f, 1.f, 1.f};
     if (p.mode == EPI_RESID && n4 + 3 < p.N) {
       const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
@@ -428,17 +459,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
           g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
           g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
         }
-        acc[u] = p.splits > 1 ? __ldcg(reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane))
-                              : *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
+        acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
         rs[u] = rstd_s[tlc];
-      }
-      for (int r = 1; r < p.splits; ++r) {                     // split order: fixed summation order
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-          const int tlc = live[u] ? tb + NW * u : tb;
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(recv + (size_t)(r * per + tlc) * TC_BLOCK_N + 4 * lane));
-          acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
-        }
       }
 #pragma unroll
       for (int u = 0; u < RB; ++u) { acc[u].x *= rs[u]; acc[u].y *= rs[u]; acc[u].z *= rs[u]; acc[u].w *= rs[u]; }
