@@ -266,11 +266,10 @@ constexpr int GEMM_MAX_SPLITS = 4;
 
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  static const int cap = getenv("BITA_SPLIT_CAP") ? atoi(getenv("BITA_SPLIT_CAP")) : GEMM_MAX_SPLITS;
   int s = GEMM_MAX_CTAS / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
-  if (s > cap) s = cap;
+  if (s > GEMM_MAX_SPLITS) s = GEMM_MAX_SPLITS;
   if (s < 1) s = 1;
   return s;
 }
@@ -334,8 +333,7 @@ void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
   if (w > 8) w = 8;
   const int rt = (M + 16 * w - 1) / (16 * w);
   const int ctas = H * B * rt;
-  static const int target = getenv("BITA_ATTN_CTAS") ? atoi(getenv("BITA_ATTN_CTAS")) : 296;
-  int s = target / ctas;                       // every slice resident at once (two CTAs per SM)
+  int s = 296 / ctas;                          // every slice resident at once (two CTAs per SM)
   if (s < 1) s = 1;
   if (s > 6) s = 6;
   *warps = w; *row_tiles = rt; *splits = s;
