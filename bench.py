@@ -362,6 +362,65 @@ def run_ours(args, shape, tmpl):
         dist.destroy_process_group()
 
 
+def run_attn_sweep():
+    """Tree-attention kernel alone: bf16 q of (1 + 4 + N) rows x 32 heads x 128 against caches of C tokens,
+    seeded random trees, batch 1 and 8.  Prints one JSON line per case (latency, KV GB/s)."""
+    from paper_2401_12522_b200 import bita_tree_attention
+    from paper_2401_12522_b200.build import build
+    build()
+    dev = torch.device("cuda:0")
+    peak, _ = _peaks()
+    H = H_kv = 32
+    D, P = 128, 16
+    for B in (1, 8):
+        for N in (16, 64, 128):
+            M = 1 + N + 4
+            tmpl = synth.random_recursive_template(N + 1, N)
+            W = (M + 31) // 32
+            depth = tmpl.depths()
+            vis = torch.zeros((M, W), dtype=torch.int64)
+            anc = [[0]]
+            for i, p_ in enumerate(tmpl.parent):
+                anc.append(anc[p_ + 1] + [i + 1])
+            rows = anc + [anc[0] + list(range(1 + N, 1 + N + i + 1)) for i in range(4)]
+            for r, cols in enumerate(rows):
+                for c in cols:
+                    vis[r, c >> 5] |= 1 << (c & 31)
+            vis = (vis & 0xFFFFFFFF).to(torch.int64)
+            vis32 = torch.where(vis >= 2 ** 31, vis - 2 ** 32, vis).to(torch.int32)
+            vis_d = vis32[None].repeat(B, 1, 1).contiguous().to(dev)
+            sp = torch.zeros((B, M), dtype=torch.uint8)
+            sp[:, 1 + N:] = 1
+            sp = sp.to(dev)
+            for C in (512, 2048, 8192, 32768):
+                C_max = C + M + 8
+                q = synth.pseudo_normal(1, 1, (B, M, H, D), 1.0, dtype=torch.bfloat16, device=dev)
+                k = synth.pseudo_normal(1, 2, (B, H_kv, C_max, D), 1.0, dtype=torch.bfloat16, device=dev)
+                v = synth.pseudo_normal(1, 3, (B, H_kv, C_max, D), 1.0, dtype=torch.bfloat16, device=dev)
+                pk = synth.pseudo_normal(1, 4, (H_kv, P, D), 1.0, dtype=torch.bfloat16, device=dev)
+                pv = synth.pseudo_normal(1, 5, (H_kv, P, D), 1.0, dtype=torch.bfloat16, device=dev)
+                ctx = torch.full((B,), C, dtype=torch.int32, device=dev)
+                out = torch.empty((B, M, H * D), dtype=torch.bfloat16, device=dev)
+                flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+                ws = None
+                times = []
+                for it in range(8):
+                    flush.zero_()                                # caches smaller than L2 would otherwise stay in it
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    bita_tree_attention(q, k, v, vis_d, pk, pv, sp, ctx, H_kv=H_kv, P=P, out=out)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        times.append(e0.elapsed_time(e1))
+                ms = statistics.median(times)
+                kv_bytes = B * 2 * (C + M) * H_kv * D * 2
+                print(json.dumps({"metric": "tree_attention_latency", "B": B, "rows": M, "C": C, "ms": ms,
+                                  "kv_gb_per_s": kv_bytes / ms / 1e6, "hbm_frac": kv_bytes / ms / 1e6 / peak,
+                                  "l2": "flushed before each launch"}))
+                del q, k, v, flush
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -373,7 +432,11 @@ def main():
     ap.add_argument("--planted", type=float, default=0.6)
     ap.add_argument("--cpu-samples", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--attn-sweep", action="store_true", help="time the tree-attention kernel alone over the sweep shapes")
     args = ap.parse_args()
+    if args.attn_sweep:
+        run_attn_sweep()
+        return
     if args.warmup < 3:
         args.warmup = 3
     shape = synth.CONFIGS[args.workload]
