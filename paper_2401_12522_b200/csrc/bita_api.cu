@@ -329,9 +329,9 @@ inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
 
 // Attention launch shape: warps per CTA, row tiles, key slices (about two CTAs per SM in total).
 void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
-  int w = (M + 15) / 16;
-  if (w > 8) w = 8;
-  const int rt = (M + 16 * w - 1) / (16 * w);
+  const int groups = (M + 15) / 16;            // 16-row groups, one warp each
+  const int rt = (groups + 7) / 8;             // at most 8 warps per CTA
+  const int w = (groups + rt - 1) / rt;        // spread evenly over the row tiles
   const int ctas = H * B * rt;
   int s = 296 / ctas;                          // every slice resident at once (two CTAs per SM)
   if (s < 1) s = 1;
