@@ -255,6 +255,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
             return true;
           }
           if (ld_acquire(cp.phase_done + ph - 1) < G) return false;
+          asm volatile("fence.proxy.async;" ::: "memory");   // other CTAs' stores, then this thread's TMA reads
           if (!waited_pdl) { pdl_wait(); waited_pdl = true; }
           return true;
         };
@@ -486,7 +487,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
         ++uc;
       }
       if (ph + 1 < cp.n_phases) {
-        // this CTA's share of the phase is written: tell the grid
+        // this CTA's share of the phase is written (and will be read by TMA): tell the grid
+        asm volatile("fence.proxy.async;" ::: "memory");
         __threadfence();
         epi_bar();
         if (tid_e == 0) atomicAdd(cp.phase_done + ph, 1);
