@@ -262,6 +262,11 @@ struct GemmDesc {
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
+// Synchronisation words of one chained launch: CH_MAX_PHASES grid-wide phase counters, then
+// CHAIN_CNT_STRIDE split counters per phase.  Zeroed once per pass, never reset by the kernels.
+constexpr int CHAIN_CNT_STRIDE = 1024;
+constexpr int CHAIN_CNT_BASE = 64;
+constexpr int CHAIN_SYNC_INTS = CHAIN_CNT_BASE + CH_MAX_PHASES * CHAIN_CNT_STRIDE;
 constexpr int GEMM_MAX_CTAS = 296;
 constexpr int GEMM_MAX_SPLITS = 4;
 
@@ -380,7 +385,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
   t.gemm_cnt = (int32_t*)take(4096 * 4);
-  t.chain_done = (int32_t*)take((size_t)(m.L + 1) * CH_MAX_PHASES * 4);
+  t.chain_done = (int32_t*)take((size_t)m.L * CHAIN_SYNC_INTS * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -477,10 +482,9 @@ struct ProjOp {
 };
 
 constexpr size_t CHAIN_SMEM_BUDGET = 110 * 1024;   // two CTAs per SM
-constexpr int CHAIN_CNT_STRIDE = 1024;             // split counters of phase i start at i * stride
 
 // Up to CH_MAX_PHASES dependent projections as one persistent kernel (chain.cuh).
-int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* phase_done) {
+int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* sync) {
   const int n_pad = pad16(M);
   const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
   const size_t xchg = (size_t)CH_XCHG_TOKENS * TC_BLOCK_N * 4;
@@ -490,6 +494,7 @@ int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* phase_do
   const size_t smem = (size_t)stages * stage + xchg + 1024;
   if (!c->chain_ctas) {
     CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BUDGET));
+    CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     int per_sm = 0, dev = 0, sms = 0;
     CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_chain, TC_THREADS, smem));
     CU_TRY(cudaGetDevice(&dev));
@@ -504,7 +509,7 @@ int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* phase_do
   ChainMaps maps;
   ChainParams cp{};
   cp.n_phases = n;
-  cp.phase_done = phase_done;
+  cp.phase_done = sync;
   for (int i = 0; i < n; ++i) {
     const GemmDesc& g = *ops[i].g;
     auto key = std::make_tuple((const void*)ops[i].X, g.K, n_pad);
@@ -537,7 +542,7 @@ int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* phase_do
     p.tmem_cols = cols;
     p.status = &c->b.state->status;
     p.part = c->b.gemm_part;
-    p.tile_counters = c->b.gemm_cnt + i * CHAIN_CNT_STRIDE;
+    p.tile_counters = sync + CHAIN_CNT_BASE + i * CHAIN_CNT_STRIDE;
     cp.ph[i] = p;
     cp.tiles[i] = g.tiles;
   }
@@ -630,7 +635,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   };
   auto single = [&](const ProjOp& o) { return gemm(c, *o.g, o.X, M, o.p); };
   const bool chained = c->chain && pad16(M) <= 96;
-  if (chained) CU_TRY(cudaMemsetAsync(b.chain_done, 0, (size_t)(m.L + 1) * CH_MAX_PHASES * 4, s));
+  if (chained) CU_TRY(cudaMemsetAsync(b.chain_done, 0, (size_t)m.L * CHAIN_SYNC_INTS * 4, s));
   if (chained && (rc = single(op_qkv(0)))) return rc;
   for (int l = 0; l < m.L; ++l) {
     bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
@@ -648,7 +653,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     c->launches += 2;
     if (chained) {
       ProjOp ops[CH_MAX_PHASES] = {op_o(l), op_gu(l), op_dn(l), op_qkv(l + 1 < m.L ? l + 1 : l)};
-      if ((rc = launch_chain(c, ops, l + 1 < m.L ? 4 : 3, M, b.chain_done + (size_t)l * CH_MAX_PHASES))) return rc;
+      if ((rc = launch_chain(c, ops, l + 1 < m.L ? 4 : 3, M, b.chain_done + (size_t)l * CHAIN_SYNC_INTS))) return rc;
     } else {
       if ((rc = single(op_o(l)))) return rc;
       if ((rc = single(op_gu(l)))) return rc;

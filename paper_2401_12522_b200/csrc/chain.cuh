@@ -12,7 +12,9 @@
 //   * two TMEM accumulators alternate, so the epilogue of one unit overlaps the MMAs of the next;
 //   * the epilogue works straight from the accumulator (thread = output feature), never touching
 //     the ring, so the producer is never blocked by it.
-// Split-K, the fused epilogues and the fixed summation order are those of gemm_tc.cuh.
+// Split-K: every split writes its partial tile, then reduces its own share of the tile's rows (in
+// split order, so the sum does not depend on timing) and applies the fused epilogue to them.  The
+// per-tile arrival counters are zero at launch and are not reset.
 #pragma once
 
 #include "gemm_tc.cuh"
@@ -61,19 +63,20 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Fused operation on 16 rows (c0 .. c0+15) of one output feature: `v[j]` is the projection result
-// of row c0+j for feature row `fr` of tile `tile`, already summed over the splits.  Called by all
-// 128 epilogue threads together (it synchronises them when values cross warps).
-__device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int fr, int lane, int c0, float* v,
-                                            const float* rstd_s, float* xchg) {
+// Fused operation on up to 16 rows (c0 .. min(c0+16, row_end)-1) of one output feature: `v[j]` is
+// the projection result of row c0+j for feature row `fr` of tile `tile`, already summed over the
+// splits.  Called by all 128 epilogue threads together (it synchronises them when values cross
+// warps).
+__device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int fr, int lane, int c0, int row_end,
+                                            float* v, const float* rstd_s, float* xchg) {
 #pragma unroll
-  for (int j = 0; j < 16; ++j) v[j] *= rstd_s[c0 + j];
+  for (int j = 0; j < 16; ++j) v[j] *= rstd_s[(c0 + j) & (BITA_MAX_ROWS - 1)];
   if (p.mode == EPI_STORE) {
     const int n = tile * TC_BLOCK_N + fr;
     if (n < p.N) {
 #pragma unroll
       for (int j = 0; j < 16; ++j)
-        if (c0 + j < p.M) p.out[(size_t)(c0 + j) * p.ldo + n] = v[j];
+        if (c0 + j < row_end) p.out[(size_t)(c0 + j) * p.ldo + n] = v[j];
     }
   } else if (p.mode == EPI_RESID) {
     const int n = tile * TC_BLOCK_N + fr;
@@ -81,10 +84,10 @@ __device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int
     const float g = valid ? bf2f(p.gain[n]) : 0.f;
     float xv[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) xv[j] = (valid && c0 + j < p.M) ? p.x[(size_t)(c0 + j) * p.N + n] : 0.f;
+    for (int j = 0; j < 16; ++j) xv[j] = (valid && c0 + j < row_end) ? p.x[(size_t)(c0 + j) * p.N + n] : 0.f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const bool live = valid && c0 + j < p.M;
+      const bool live = valid && c0 + j < row_end;
       xv[j] += v[j];
       if (live) {
         p.x[(size_t)(c0 + j) * p.N + n] = xv[j];
@@ -100,7 +103,7 @@ __device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int
     if (lane == 0) {
 #pragma unroll
       for (int j = 0; j < 16; ++j)
-        if (c0 + j < p.M) atomicAdd(p.out_sumsq + c0 + j, sumsq_to_fixed(xv[j]));
+        if (c0 + j < row_end) atomicAdd(p.out_sumsq + c0 + j, sumsq_to_fixed(xv[j]));
     }
   } else if (p.mode == EPI_SWIGLU) {
     // tile rows 0..63 are gate features, rows 64..127 the matching up features
@@ -117,7 +120,7 @@ __device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int
         for (int j = 0; j < CH_XCHG_TOKENS; ++j) {
           const int tok = c0 + r8 * 8 + j;
           const float gt = v[r8 * 8 + j], up = xchg[j * 64 + fr];
-          if (tok < p.M) p.hf[(size_t)tok * p.F + f] = f2bf(__fdividef(gt, 1.0f + __expf(-gt)) * up);
+          if (tok < row_end) p.hf[(size_t)tok * p.F + f] = f2bf(__fdividef(gt, 1.0f + __expf(-gt)) * up);
         }
       }
       epi_bar();
@@ -134,7 +137,7 @@ __device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int
     const int C = *p.len_ptr;
     bf16* dst = nullptr;
     size_t stride = 0;
-    int t_end = p.M;
+    int t_end = row_end;
     if (valid) {
       if (head < p.H) {
         dst = p.q + (size_t)head * p.D + dd;
@@ -144,7 +147,7 @@ __device__ __forceinline__ void chain_apply(const GemmTcParams& p, int tile, int
                                          : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
         dst = base + (size_t)C * p.D + dd;
         stride = p.D;
-        t_end = min(p.M, p.C_max - C);                         // never write past the cache
+        t_end = min(row_end, p.C_max - C);                         // never write past the cache
       }
     }
 #pragma unroll
@@ -182,7 +185,6 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
   __shared__ __align__(8) uint64_t bar_tempty[2];    // accumulator buffer b read out
   __shared__ uint32_t tmem_base_slot;
   __shared__ float rstd_s[BITA_MAX_ROWS];
-  __shared__ int last_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -430,7 +432,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
               tc_fence_before();
               mbar_arrive(smem_u32(&bar_tempty[buf]));
             }
-            chain_apply(p, cu.tile, fr, lane, c, v, rstd_s, xchg);
+            chain_apply(p, cu.tile, fr, lane, c, p.M, v, rstd_s, xchg);
           }
         } else {
           const size_t tile_elems = (size_t)p.M * TC_BLOCK_N;
@@ -452,37 +454,46 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
           mbar_arrive(smem_u32(&bar_tempty[buf]));
           __threadfence();
           epi_bar();
-          if (tid_e == 0) {
-            const int old = atomicAdd(p.tile_counters + cu.tile, 1);
-            last_flag = old == p.splits - 1;
-            if (last_flag) p.tile_counters[cu.tile] = 0;
-          }
-          epi_bar();
-          if (last_flag) {
-            __threadfence();
-            for (int c = 0; c < n_pad; c += 16) {
-              float v[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) v[j] = 0.f;
-              for (int r0 = 0; r0 < p.splits; r0 += 4) {       // four partial tiles' loads in flight together
-                float t[4][16];
-#pragma unroll
-                for (int rr = 0; rr < 4; ++rr) {
-                  const float* src = part_tile + (size_t)(r0 + rr) * tile_elems + fr;
-#pragma unroll
-                  for (int j = 0; j < 16; ++j)
-                    t[rr][j] = (r0 + rr < p.splits && c + j < p.M) ? __ldcg(src + (c + j) * TC_BLOCK_N) : 0.f;
-                }
-#pragma unroll
-                for (int rr = 0; rr < 4; ++rr) {               // split order: fixed summation order
-#pragma unroll
-                  for (int j = 0; j < 16; ++j) v[j] += t[rr][j];
-                }
+          if (tid_e == 0) atomicAdd(p.tile_counters + cu.tile, 1);
+          // Every split of the tile reduces its own share of the rows once all partial tiles are
+          // there: the other splits run on resident CTAs that reach this point without waiting
+          // for this one (units are taken in (tile, split) order), so the wait is short and bounded.
+          {
+            unsigned long long t0 = 0;
+            uint32_t spin = 0;
+            while (ok && ld_acquire(p.tile_counters + cu.tile) < p.splits) {
+              if ((++spin & 63u) == 0) {
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > TC_WAIT_LIMIT_NS) { ok = false; atomicExch(status, BITA_ERR_TIMEOUT); }
               }
-              chain_apply(p, cu.tile, fr, lane, c, v, rstd_s, xchg);
             }
           }
-          epi_bar();
+          const int r_begin = (int)((long)p.M * cu.split / p.splits);
+          const int r_end = (int)((long)p.M * (cu.split + 1) / p.splits);
+          const int chunk = p.splits > 4 ? 8 : 16;               // at most 64 loads in flight per thread
+          for (int c = r_begin; c < r_end; c += chunk) {
+            const int c_end = min(r_end, c + chunk);
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = 0.f;
+            for (int q0 = 0; q0 < p.splits; q0 += 4) {
+              float t[4][16];
+#pragma unroll
+              for (int rr = 0; rr < 4; ++rr) {
+                const float* src = part_tile + (size_t)(q0 + rr) * tile_elems + fr;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  t[rr][j] = (ok && q0 + rr < p.splits && c + j < c_end) ? __ldcg(src + (c + j) * TC_BLOCK_N) : 0.f;
+              }
+#pragma unroll
+              for (int rr = 0; rr < 4; ++rr) {                   // split order: fixed summation order
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += t[rr][j];
+              }
+            }
+            chain_apply(p, cu.tile, fr, lane, c, c_end, v, rstd_s, xchg);
+          }
         }
         ++uc;
       }
