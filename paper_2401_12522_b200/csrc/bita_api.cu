@@ -495,12 +495,21 @@ int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* sync) {
   if (!c->chain_ctas) {
     CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BUDGET));
     CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-    int per_sm = 0, dev = 0, sms = 0;
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_chain, TC_THREADS, smem));
+    // Two CTAs share an SM: 168 registers x 192 threads and under 112 KB of shared memory each,
+    // 2 x tmem_cols <= 512 TMEM columns.  (The occupancy query of the runtime answers 1 for every
+    // kernel that allocates tensor memory, whatever its footprint; k_gemm_tc with the same
+    // footprint is seen running two per SM, so the count is taken from the resources.)
+    int per_sm = 2, dev = 0, sms = 0;
+    cudaFuncAttributes fa;
+    CU_TRY(cudaFuncGetAttributes(&fa, k_chain));
     CU_TRY(cudaGetDevice(&dev));
     CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if (per_sm < 1 || sms < 1) return BITA_ERR_CUDA;
-    if (per_sm > 2) per_sm = 2;
+    int smem_sm = 0, regs_sm = 0;
+    CU_TRY(cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
+    CU_TRY(cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev));
+    const size_t per_cta_smem = CHAIN_SMEM_BUDGET + fa.sharedSizeBytes + 1024;
+    if (2 * per_cta_smem > (size_t)smem_sm || 2 * fa.numRegs * TC_THREADS > regs_sm) per_sm = 1;
+    if (sms < 1) return BITA_ERR_CUDA;
     c->chain_ctas = per_sm * sms;
   }
   const int G = c->chain_ctas;
