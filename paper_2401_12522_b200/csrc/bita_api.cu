@@ -275,7 +275,8 @@ int gemm_splits(int tiles, int K, int max_splits) {
   int s = GEMM_MAX_CTAS / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
-  if (s > GEMM_MAX_SPLITS) s = GEMM_MAX_SPLITS;
+  static const int cap = getenv("BITA_MAX_SPLITS") ? atoi(getenv("BITA_MAX_SPLITS")) : GEMM_MAX_SPLITS;
+  if (s > cap) s = cap;
   if (s < 1) s = 1;
   return s;
 }

@@ -52,11 +52,6 @@ __device__ __forceinline__ ChainUnit chain_unit(const GemmTcParams& p, int u) {
   return r;
 }
 
-__device__ __forceinline__ int ld_acquire(const int32_t* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -256,7 +251,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
             waited_pdl = true;
             return true;
           }
-          if (ld_acquire(cp.phase_done + ph - 1) < G) return false;
+          if (ld_acquire_gpu(cp.phase_done + ph - 1) < G) return false;
           asm volatile("fence.proxy.async;" ::: "memory");   // other CTAs' stores, then this thread's TMA reads
           if (!waited_pdl) { pdl_wait(); waited_pdl = true; }
           return true;
@@ -405,7 +400,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
           if (ph > 0) {
             unsigned long long t0 = 0;
             uint32_t spin = 0;
-            while (ok && ld_acquire(cp.phase_done + ph - 1) < G) {
+            while (ok && ld_acquire_gpu(cp.phase_done + ph - 1) < G) {
               if ((++spin & 63u) == 0) {
                 const unsigned long long now = global_ns();
                 if (t0 == 0) t0 = now;
@@ -461,7 +456,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) k_chain(const __grid_constant__
           {
             unsigned long long t0 = 0;
             uint32_t spin = 0;
-            while (ok && ld_acquire(p.tile_counters + cu.tile) < p.splits) {
+            while (ok && ld_acquire_gpu(p.tile_counters + cu.tile) < p.splits) {
               if ((++spin & 63u) == 0) {
                 const unsigned long long now = global_ns();
                 if (t0 == 0) t0 = now;

@@ -35,6 +35,7 @@ constexpr int TC_BLOCK_N = 128;   // weight rows per tile (MMA M)
 constexpr int TC_BLOCK_K = 64;    // bf16 elements per K block = 128 bytes = one swizzle row
 constexpr int TC_UMMA_K = 16;
 constexpr int TC_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr int TC_DEPART_OFFSET = 2048;     // tile_counters: [0, 2048) arrivals, [2048, 4096) departures
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // a wait that lasts 2 s has failed
 
 enum GemmEpilogue : int32_t {
@@ -71,7 +72,7 @@ struct GemmTcParams {
   int32_t mode;          // GemmEpilogue
   int32_t* status;       // device status word (sticky error flag)
   float* part;           // split-K exchange buffer [tiles][splits][M][128] fp32 (splits > 1)
-  int32_t* tile_counters;  // [tiles], zero before the launch; left zero by the kernel
+  int32_t* tile_counters;  // [4096]: arrivals per tile, then (at TC_DEPART_OFFSET) departures; zero before the launch, left zero
   // row scale of the input (RMSNorm statistics of the rows of X), or null: y *= rstd(row)
   const unsigned long long* in_sumsq;
   int32_t norm_d;
@@ -120,6 +121,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status) {
   unsigned long long t0 = 0;
@@ -216,7 +222,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t bar_acc;
   __shared__ uint32_t tmem_base_slot;
   __shared__ float rstd_s[BITA_MAX_ROWS];
-  __shared__ int last_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -330,10 +335,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   // splits == 1: the tile goes to shared memory (`stg`, the pipeline stages, free once the
   //              accumulator barrier has completed), row-major [M][128] fp32.
   // splits  > 1: every split stores its partial tile to the global exchange buffer
-  //              part[tile][split][M][128] (L2-resident, overwritten by every projection), then
-  //              bumps the tile's counter; the split that finds the counter complete sums the
-  //              partial tiles, always in split order, and applies the fused operation.  No CTA
-  //              ever waits for another, and the early leavers free their SM for the next kernel.
+  //              part[tile][split][M][128] (L2-resident, overwritten by every projection) and
+  //              counts itself in; once all splits of the tile are in, each of them sums an equal
+  //              share of the rows over the partial tiles, always in split order, and applies
+  //              the fused operation to those rows.
   float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
   const size_t tile_elems = (size_t)p.M * TC_BLOCK_N;
   float* part_tile = p.part + (size_t)tile * p.splits * tile_elems;      // this tile's partials, split-major
@@ -366,61 +371,79 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   }
   tc_fence_before();
   __syncthreads();
-  bool reducer = true;
+  // Rows of the tile this CTA finishes: all of them without a split, else an equal share, so that
+  // the reduction and the fused operation of a tile are spread over all its splits.
+  const int t0 = p.splits > 1 ? (int)((long)p.M * split / p.splits) : 0;
+  const int cnt = (p.splits > 1 ? (int)((long)p.M * (split + 1) / p.splits) : p.M) - t0;
   if (p.splits > 1) {
+    int32_t* arrived = p.tile_counters + tile;
+    int32_t* departed = p.tile_counters + TC_DEPART_OFFSET + tile;
     if (threadIdx.x == 0) {
-      const int old = atomicAdd(p.tile_counters + tile, 1);
-      last_flag = old == p.splits - 1;
-      if (last_flag) p.tile_counters[tile] = 0;                // ready for the next projection
+      // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
+      // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+      atomicAdd(arrived, 1);
+      unsigned long long w0 = 0;
+      bool ok = true;
+      for (uint32_t spin = 0; ld_acquire_gpu(arrived) < p.splits; ++spin) {
+        if ((spin & 63u) == 63u) {
+          const unsigned long long now = global_ns();
+          if (w0 == 0) w0 = now;
+          else if (now - w0 > TC_WAIT_LIMIT_NS) { ok = false; break; }
+        }
+      }
+      if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
+      __threadfence();
     }
     __syncthreads();
-    reducer = last_flag != 0;
-    if (reducer) {
-      __threadfence();
-      // Sum the partial tiles into `stg`, in split order.  Each thread takes 16-byte items of the
-      // tile; the loads of four items (all their splits) are in flight together.
-      const int items = p.M * (TC_BLOCK_N / 4);
-      const float4* src = reinterpret_cast<const float4*>(part_tile);
-      const int stride4 = (int)(tile_elems / 4);               // between the splits' tiles
-      for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
+    // Sum rows t0 .. t0+cnt of the partial tiles into `stg` (local row order), in split order.  A
+    // thread takes 16-byte items; the loads of four items (four splits each) fly together.
+    const int items = cnt * (TC_BLOCK_N / 4);
+    const float4* src = reinterpret_cast<const float4*>(part_tile) + (size_t)t0 * (TC_BLOCK_N / 4);
+    const int stride4 = (int)(tile_elems / 4);               // between the splits' tiles
+    for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
+      float4 a4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) a4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int r0 = 0; r0 < p.splits; r0 += 4) {
         float4 v[4][4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int i = min(i0 + u * TC_THREADS, items - 1);
 #pragma unroll
           for (int r = 0; r < 4; ++r)
-            if (r < p.splits) v[u][r] = __ldcg(src + (size_t)r * stride4 + i);
+            if (r0 + r < p.splits) v[u][r] = __ldcg(src + (size_t)(r0 + r) * stride4 + i);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const int i = i0 + u * TC_THREADS;
-          float4 a4 = v[u][0];
 #pragma unroll
-          for (int r = 1; r < 4; ++r)
-            if (r < p.splits) { a4.x += v[u][r].x; a4.y += v[u][r].y; a4.z += v[u][r].z; a4.w += v[u][r].w; }
-          for (int r = 4; r < p.splits; ++r) {                 // more than four splits: the rest one by one
-            const float4 w = __ldcg(src + (size_t)r * stride4 + min(i, items - 1));
-            a4.x += w.x; a4.y += w.y; a4.z += w.z; a4.w += w.w;
-          }
-          if (i < items) reinterpret_cast<float4*>(stg)[i] = a4;
+          for (int r = 0; r < 4; ++r)
+            if (r0 + r < p.splits) { a4[u].x += v[u][r].x; a4[u].y += v[u][r].y; a4[u].z += v[u][r].z; a4[u].w += v[u][r].w; }
         }
       }
-      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * TC_THREADS;
+        if (i < items) reinterpret_cast<float4*>(stg)[i] = a4[u];
+      }
+    }
+    __syncthreads();
+    // The partial tiles are read: the last split to say so leaves both counters at zero for the
+    // next projection (which touches them only after this kernel has completed).
+    if (threadIdx.x == 0) {
+      const int old = atomicAdd(departed, 1);
+      if (old == p.splits - 1) { *arrived = 0; *departed = 0; }
     }
   }
   const float* recv = stg;
-  const int per = p.M;
-  const int rank = 0;
 
   // ---------------- epilogue, part 2: reduction over the splits + fused operation, all six warps.
   // A thread handles 4 consecutive features (quad = lane) of one row at a time; the warps take
   // rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 (or 32)
   // features away, i.e. 16 (or 8) lanes, and are exchanged with a warp shuffle.
-  if (reducer) {
+  {
     constexpr int RB = 6;                                      // rows per batch: their global loads fly together
     constexpr int NW = TC_THREADS / 32;
     pdl_wait();
-    const int t0 = rank * per, cnt = min(p.M, t0 + per) - t0;  // rows owned by this split
     const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
     const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
     float g4[4] = {1.f, 1.f, 1.f, 1.f};
@@ -460,7 +483,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
           g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
         }
         acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
-        rs[u] = rstd_s[tlc];
+        rs[u] = rstd_s[t0 + tlc];
       }
 #pragma unroll
       for (int u = 0; u < RB; ++u) { acc[u].x *= rs[u]; acc[u].y *= rs[u]; acc[u].z *= rs[u]; acc[u].w *= rs[u]; }
