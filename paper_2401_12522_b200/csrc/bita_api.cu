@@ -11,7 +11,6 @@
 #include <vector>
 
 #include "attention_tc.cuh"
-#include "chain.cuh"
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "step_kernels.cuh"
@@ -262,21 +261,15 @@ struct GemmDesc {
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
-// Synchronisation words of one chained launch: CH_MAX_PHASES grid-wide phase counters, then
-// CHAIN_CNT_STRIDE split counters per phase.  Zeroed once per pass, never reset by the kernels.
-constexpr int CHAIN_CNT_STRIDE = 1024;
-constexpr int CHAIN_CNT_BASE = 64;
-constexpr int CHAIN_SYNC_INTS = CHAIN_CNT_BASE + CH_MAX_PHASES * CHAIN_CNT_STRIDE;
 constexpr int GEMM_MAX_CTAS = 296;
-constexpr int GEMM_MAX_SPLITS = 4;
+constexpr int GEMM_MAX_SPLITS = 8;
 
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
   int s = GEMM_MAX_CTAS / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
-  static const int cap = getenv("BITA_MAX_SPLITS") ? atoi(getenv("BITA_MAX_SPLITS")) : GEMM_MAX_SPLITS;
-  if (s > cap) s = cap;
+  if (s > GEMM_MAX_SPLITS) s = GEMM_MAX_SPLITS;
   if (s < 1) s = 1;
   return s;
 }
@@ -355,7 +348,7 @@ int attn_splits(int H, int B, int M) {
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
-  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt; int32_t* chain_done;
+  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
 };
@@ -386,7 +379,6 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
   t.gemm_cnt = (int32_t*)take(4096 * 4);
-  t.chain_done = (int32_t*)take((size_t)m.L * CHAIN_SYNC_INTS * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -418,8 +410,7 @@ struct bita_ctx {
   GemmDesc d_head;
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
   bool pdl;                             // programmatic dependent launch between the kernels of a pass
-  bool chain;                           // O / gate-up / down / next q-k-v as phases of one persistent kernel
-  int chain_ctas;                       // resident CTAs of that kernel (0 = not yet asked)
+
   // optional per-family event timing
   bool timing;
   std::vector<cudaEvent_t> ev;          // pairs (start, stop)
@@ -473,96 +464,6 @@ GemmTcParams epi_store(float* out, int ldo) {
   GemmTcParams p{};
   p.mode = EPI_STORE; p.out = out; p.ldo = ldo;
   return p;
-}
-
-// One projection of a pass: weights, activation buffer, epilogue.
-struct ProjOp {
-  const GemmDesc* g;
-  const bf16* X;
-  GemmTcParams p;
-};
-
-constexpr size_t CHAIN_SMEM_BUDGET = 110 * 1024;   // two CTAs per SM
-
-// Up to CH_MAX_PHASES dependent projections as one persistent kernel (chain.cuh).
-int launch_chain(bita_ctx* c, const ProjOp* ops, int n, int M, int32_t* sync) {
-  const int n_pad = pad16(M);
-  const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  const size_t xchg = (size_t)CH_XCHG_TOKENS * TC_BLOCK_N * 4;
-  int stages = (int)((CHAIN_SMEM_BUDGET - 1024 - xchg) / stage);
-  if (stages > 10) stages = 10;
-  if (stages < 2) return BITA_ERR_INVALID_ARG;
-  const size_t smem = (size_t)stages * stage + xchg + 1024;
-  if (!c->chain_ctas) {
-    CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BUDGET));
-    CU_TRY(cudaFuncSetAttribute(k_chain, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-    // Two CTAs share an SM: 168 registers x 192 threads and under 112 KB of shared memory each,
-    // 2 x tmem_cols <= 512 TMEM columns.  (The occupancy query of the runtime answers 1 for every
-    // kernel that allocates tensor memory, whatever its footprint; k_gemm_tc with the same
-    // footprint is seen running two per SM, so the count is taken from the resources.)
-    int per_sm = 2, dev = 0, sms = 0;
-    cudaFuncAttributes fa;
-    CU_TRY(cudaFuncGetAttributes(&fa, k_chain));
-    CU_TRY(cudaGetDevice(&dev));
-    CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    int smem_sm = 0, regs_sm = 0;
-    CU_TRY(cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
-    CU_TRY(cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev));
-    const size_t per_cta_smem = CHAIN_SMEM_BUDGET + fa.sharedSizeBytes + 1024;
-    if (2 * per_cta_smem > (size_t)smem_sm || 2 * fa.numRegs * TC_THREADS > regs_sm) per_sm = 1;
-    if (sms < 1) return BITA_ERR_CUDA;
-    c->chain_ctas = per_sm * sms;
-  }
-  const int G = c->chain_ctas;
-  int cols = 32;
-  while (cols < 2 * n_pad) cols <<= 1;
-  ChainMaps maps;
-  ChainParams cp{};
-  cp.n_phases = n;
-  cp.phase_done = sync;
-  for (int i = 0; i < n; ++i) {
-    const GemmDesc& g = *ops[i].g;
-    auto key = std::make_tuple((const void*)ops[i].X, g.K, n_pad);
-    auto it = c->act_maps.find(key);
-    if (it == c->act_maps.end()) {
-      CUtensorMap m;
-      int rc = make_map(&m, ops[i].X, g.K, BITA_MAX_ROWS, n_pad);
-      if (rc) return rc;
-      it = c->act_maps.emplace(key, m).first;
-    }
-    maps.a0[i] = g.a0;
-    maps.a1[i] = g.a1;
-    maps.b[i] = it->second;
-    GemmTcParams p = ops[i].p;
-    const int kb = (g.K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-    if (g.tiles > CHAIN_CNT_STRIDE) return BITA_ERR_INVALID_ARG;
-    // Units (tile, split) go round-robin over the G resident CTAs.  The busiest CTA gets
-    // ceil(units / G) units of ceil(kb / s) K blocks each, plus a fixed cost per unit (partial tile
-    // out) and per split (partial tiles back in), counted in K-block times.
-    int splits = 1;
-    long best = -1;
-    const long cap_units = (long)GEMM_MAX_CTAS * BITA_MAX_ROWS / M;         // room for partial tiles
-    for (int sp = 1; sp <= 8; ++sp) {
-      if (sp > 1 && (kb / sp < 4 || (long)g.tiles * sp > cap_units)) break;
-      const long per_cta = ((long)g.tiles * sp + G - 1) / G;
-      const long cost = per_cta * ((kb + sp - 1) / sp + 3) + sp;
-      if (best < 0 || cost < best) { best = cost; splits = sp; }
-    }
-    p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.stages = stages; p.splits = splits; p.dual = g.dual;
-    p.tmem_cols = cols;
-    p.status = &c->b.state->status;
-    p.part = c->b.gemm_part;
-    p.tile_counters = sync + CHAIN_CNT_BASE + i * CHAIN_CNT_STRIDE;
-    cp.ph[i] = p;
-    cp.tiles[i] = g.tiles;
-  }
-  for (int i = n; i < CH_MAX_PHASES; ++i) {
-    maps.a0[i] = maps.a0[0]; maps.a1[i] = maps.a1[0]; maps.b[i] = maps.b[0];
-  }
-  Timed t(c, 0);
-  int rc = launch(c->stream, c->pdl, dim3(G), dim3(TC_THREADS), smem, 1, k_chain, maps, cp);
-  c->launches++;
-  return rc;
 }
 
 // Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches slices + merge.
@@ -625,6 +526,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     p.mode = EPI_RESID; p.x = b.x; p.xhat = b.xn; p.gain = (const bf16*)gain; p.out_sumsq = slot(out_slot);
     return p;
   };
+  struct ProjOp { const GemmDesc* g; const bf16* X; GemmTcParams p; };
   auto op_qkv = [&](int l) {
     GemmTcParams p{};
     p.mode = EPI_QKV; p.q = b.q; p.kc = (bf16*)kv->k + (size_t)l * layer_kv; p.vc = (bf16*)kv->v + (size_t)l * layer_kv;
@@ -644,13 +546,10 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     return ProjOp{&c->d_dn[l], b.hf, epi_resid(g_next, 2 * l + 2)};
   };
   auto single = [&](const ProjOp& o) { return gemm(c, *o.g, o.X, M, o.p); };
-  const bool chained = c->chain && pad16(M) <= 96;
-  if (chained) CU_TRY(cudaMemsetAsync(b.chain_done, 0, (size_t)m.L * CHAIN_SYNC_INTS * 4, s));
-  if (chained && (rc = single(op_qkv(0)))) return rc;
   for (int l = 0; l < m.L; ++l) {
     bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
     bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
-    if (!chained && (rc = single(op_qkv(l)))) return rc;
+    if ((rc = single(op_qkv(l)))) return rc;
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
@@ -661,14 +560,9 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
       if ((rc = launch_attention(a, pdl, s))) return rc;
     }
     c->launches += 2;
-    if (chained) {
-      ProjOp ops[CH_MAX_PHASES] = {op_o(l), op_gu(l), op_dn(l), op_qkv(l + 1 < m.L ? l + 1 : l)};
-      if ((rc = launch_chain(c, ops, l + 1 < m.L ? 4 : 3, M, b.chain_done + (size_t)l * CHAIN_SYNC_INTS))) return rc;
-    } else {
-      if ((rc = single(op_o(l)))) return rc;
-      if ((rc = single(op_gu(l)))) return rc;
-      if ((rc = single(op_dn(l)))) return rc;
-    }
+    if ((rc = single(op_o(l)))) return rc;
+    if ((rc = single(op_gu(l)))) return rc;
+    if ((rc = single(op_dn(l)))) return rc;
     if (c->dbg)
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)l * BITA_MAX_ROWS * m.d, b.x, (size_t)M * m.d * 4,
                              cudaMemcpyDeviceToDevice, s));
@@ -760,8 +654,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   c->launches = 0;
   c->timing = false;
   c->pdl = getenv("BITA_NO_PDL") == nullptr;
-  c->chain = getenv("BITA_NO_CHAIN") == nullptr;
-  c->chain_ctas = 0;
+
   c->prefilled = false;
   c->len_upper = 0;
   auto fail = [&](int code) { if (c->rec_host) cudaFreeHost(c->rec_host); delete c; return code; };
