@@ -7,8 +7,11 @@
 // `S` slices.  One CTA = one query head x one slice x up to 128 query rows; each warp owns 16 rows
 // and keeps their running maximum, running sum and output accumulator in registers (online
 // softmax, quad shuffles for the row reductions), K/V chunks are double-buffered in shared memory
-// with cp.async, Q.K^T and P.V run as bf16 m16n8k16 MMAs with fp32 accumulation.  Slices are
-// merged by k_attn_merge in slice order.
+// with cp.async, Q.K^T and P.V run as bf16 m16n8k16 MMAs with fp32 accumulation.  A single slice
+// writes the output itself.  Several slices leave partial results (running maximum, running sum,
+// unnormalised output) that are merged in slice order: inside the kernel when all CTAs of the
+// launch are resident together (`sync` given: each slice merges an equal share of its row tile's
+// rows once all slices of the tile have arrived), else by k_attn_merge.
 #pragma once
 
 #include "common.cuh"
@@ -33,7 +36,61 @@ struct AttnArgs {
   int32_t warps;             // warps per CTA = min(8, ceil(M / 16))
   int32_t row_tiles;         // ceil(M / (16 * warps))
   float scale_log2;          // log2(e) / sqrt(D)
+  int32_t* sync;             // in-kernel merge: [2][B*H*row_tiles] arrival / departure counters, zero
+                             // before the launch and left zero; null = partial results only
+  int32_t* status;           // sticky error word for a wait that ran out (may be null)
 };
+
+constexpr unsigned long long ATT_WAIT_LIMIT_NS = 2000000000ull;
+
+// Merged, normalised output of one row from its S partial results (slice order).  `lane` owns
+// D / 32 consecutive features.
+template <int D>
+__device__ __forceinline__ void attn_merge_row(const AttnArgs& a, int b, int h, int gr, int lane) {
+  constexpr int VW = D / 32;
+  const size_t p0 = (((size_t)b * a.H + h) * a.S) * a.M + gr;
+  float ms[8], ls[8], v[8][VW];
+#pragma unroll
+  for (int s = 0; s < 8; ++s) {
+    if (s < a.S) {
+      const size_t pi = p0 + (size_t)s * a.M;
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + pi * 2));
+      ms[s] = ml.x;
+      ls[s] = ml.y;
+      if (VW == 4) {
+        const float4 t = __ldcg(reinterpret_cast<const float4*>(a.part_acc + pi * D) + lane);
+        v[s][0] = t.x; v[s][1] = t.y; v[s][VW - 2] = t.z; v[s][VW - 1] = t.w;
+      } else {
+        const float2 t = __ldcg(reinterpret_cast<const float2*>(a.part_acc + pi * D) + lane);
+        v[s][0] = t.x; v[s][1] = t.y;
+      }
+    } else {
+      ms[s] = -INFINITY;
+      ls[s] = 0.f;
+#pragma unroll
+      for (int e = 0; e < VW; ++e) v[s][e] = 0.f;
+    }
+  }
+  float mx = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < 8; ++s) mx = fmaxf(mx, ms[s]);
+  float l = 0.f, o[VW];
+#pragma unroll
+  for (int e = 0; e < VW; ++e) o[e] = 0.f;
+#pragma unroll
+  for (int s = 0; s < 8; ++s) {
+    if (ms[s] == -INFINITY) continue;
+    const float w = exp2f(ms[s] - mx);
+    l += ls[s] * w;
+#pragma unroll
+    for (int e = 0; e < VW; ++e) o[e] += v[s][e] * w;
+  }
+  const float inv = l > 0.f ? 1.0f / l : 0.f;
+  bf16* dst = a.out + (((size_t)b * a.M + gr) * a.H + h) * D + lane * VW;
+#pragma unroll
+  for (int e = 0; e < VW; e += 2)
+    *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
+}
 
 constexpr int ATT_KEYS = 64;   // keys per chunk
 
@@ -269,12 +326,29 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
   }
   cp_async_wait<0>();
 
-  // ---- partial results of this slice
   l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
   l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
   l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
   l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
   const int gr_a = row0 + lr_a, gr_b = row0 + lr_b;
+  if (a.S == 1) {
+    // ---- the only slice: normalise and write the output
+    const float inv_a = l_a > 0.f ? 1.0f / l_a : 0.f, inv_b = l_b > 0.f ? 1.0f / l_b : 0.f;
+    if (gr_a < a.M) {
+      bf16* dst = a.out + (((size_t)b * a.M + gr_a) * a.H + h) * D;
+#pragma unroll
+      for (int j = 0; j < NT_O; ++j)
+        *reinterpret_cast<__nv_bfloat162*>(dst + j * 8 + 2 * t) = __floats2bfloat162_rn(o[j][0] * inv_a, o[j][1] * inv_a);
+    }
+    if (gr_b < a.M) {
+      bf16* dst = a.out + (((size_t)b * a.M + gr_b) * a.H + h) * D;
+#pragma unroll
+      for (int j = 0; j < NT_O; ++j)
+        *reinterpret_cast<__nv_bfloat162*>(dst + j * 8 + 2 * t) = __floats2bfloat162_rn(o[j][2] * inv_b, o[j][3] * inv_b);
+    }
+    return;
+  }
+  // ---- partial results of this slice
   const size_t pbase = (((size_t)b * a.H + h) * a.S + s) * a.M;
   if (gr_a < a.M) {
     if (t == 0) { a.part_ml[(pbase + gr_a) * 2] = m_a; a.part_ml[(pbase + gr_a) * 2 + 1] = l_a; }
@@ -287,6 +361,42 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
     float* dst = a.part_acc + (pbase + gr_b) * D;
 #pragma unroll
     for (int j = 0; j < NT_O; ++j) *reinterpret_cast<float2*>(dst + j * 8 + 2 * t) = make_float2(o[j][2], o[j][3]);
+  }
+  if (!a.sync) return;                                          // k_attn_merge follows
+
+  // ---- merge inside the kernel: all slices of this (sequence, head, row tile) are resident CTAs,
+  // none of which waits before its partial results are out, so the wait ends; bounded all the same.
+  const int n_sync = a.B * a.H * a.row_tiles;
+  int32_t* arrived = a.sync + ((size_t)b * a.H + h) * a.row_tiles + rt;
+  int32_t* departed = arrived + n_sync;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    atomicAdd(arrived, 1);
+    unsigned long long w0 = 0;
+    bool ok = true;
+    for (uint32_t spin = 0;; ++spin) {
+      int seen;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(arrived) : "memory");
+      if (seen >= a.S) break;
+      if ((spin & 63u) == 63u) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (w0 == 0) w0 = now;
+        else if (now - w0 > ATT_WAIT_LIMIT_NS) { ok = false; break; }
+      }
+    }
+    if (!ok && a.status) atomicExch(a.status, BITA_ERR_TIMEOUT);
+    __threadfence();
+  }
+  __syncthreads();
+  const int rows_here = min(rows_cta, a.M - row0);              // valid rows of this row tile
+  const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
+  for (int r = r_lo + warp; r < r_hi; r += a.warps) attn_merge_row<D>(a, b, h, row0 + r, lane);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int old = atomicAdd(departed, 1);
+    if (old == a.S - 1) { *arrived = 0; *departed = 0; }         // ready for the next launch
   }
 }
 

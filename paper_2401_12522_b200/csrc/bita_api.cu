@@ -261,6 +261,8 @@ struct GemmDesc {
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
+constexpr int ATTN_SYNC_SLOTS = 2048;   // (sequence, head, row tile) triples with counters for the in-kernel merge
+constexpr size_t ATTN_SYNC_BYTES = 2 * ATTN_SYNC_SLOTS * 4;
 constexpr int GEMM_MAX_CTAS = 296;
 constexpr int GEMM_MAX_SPLITS = 8;
 
@@ -348,7 +350,7 @@ int attn_splits(int H, int B, int M) {
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
-  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt;
+  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt; int32_t* attn_sync;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
 };
@@ -379,6 +381,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
   t.gemm_cnt = (int32_t*)take(4096 * 4);
+  t.attn_sync = (int32_t*)take(ATTN_SYNC_BYTES);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -466,8 +469,10 @@ GemmTcParams epi_store(float* out, int ldo) {
   return p;
 }
 
-// Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches slices + merge.
-int launch_attention(AttnArgs a, bool pdl, cudaStream_t s) {
+
+// Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches the slices (and the
+// merge kernel where the slices cannot merge themselves).
+int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched) {
   attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const int rows_cta = a.warps * 16;
@@ -483,16 +488,22 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s) {
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
   const dim3 blk(a.warps * 32);
+  // The slices merge inside the kernel when they all run in one wave (two CTAs per SM for blocks of
+  // up to five warps, one otherwise); a single slice writes the output itself.
+  const int wave = a.warps <= 5 ? 296 : 148;
+  if (a.S == 1 || a.H * a.S * a.B * a.row_tiles > wave || a.B * a.H * a.row_tiles > ATTN_SYNC_SLOTS) a.sync = nullptr;
+  const bool merge_after = a.S > 1 && !a.sync;
+  if (n_launched) *n_launched = merge_after ? 2 : 1;
   int rc;
   if (a.D == 128) {
     rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 5>, a)
                       : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 8>, a);
-    if (rc) return rc;
+    if (rc || !merge_after) return rc;
     return launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a);
   }
   rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 5>, a)
                     : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 8>, a);
-  if (rc) return rc;
+  if (rc || !merge_after) return rc;
   return launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
 
@@ -555,11 +566,13 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
+    a.sync = b.attn_sync; a.status = &b.state->status;
     {
       Timed t(c, 1);
-      if ((rc = launch_attention(a, pdl, s))) return rc;
+      int n = 0;
+      if ((rc = launch_attention(a, pdl, s, &n))) return rc;
+      c->launches += n;
     }
-    c->launches += 2;
     if ((rc = single(op_o(l)))) return rc;
     if ((rc = single(op_gu(l)))) return rc;
     if ((rc = single(op_dn(l)))) return rc;
@@ -690,6 +703,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
   if (cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  if (cudaMemsetAsync(c->b.attn_sync, 0, ATTN_SYNC_BYTES, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
@@ -884,7 +898,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
   if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
   const size_t S = attn_splits(H, B, M);
-  *out_bytes = align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
+  *out_bytes = align_up(ATTN_SYNC_BYTES) + align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
   return BITA_OK;
 }
 
@@ -904,10 +918,13 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
   a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
-  a.part_ml = (float*)workspace;
-  a.part_acc = (float*)((uint8_t*)workspace + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
+  // workspace: merge counters (zero at launch: cleared here, in stream order), then the partial results
+  CU_TRY(cudaMemsetAsync(workspace, 0, ATTN_SYNC_BYTES, (cudaStream_t)cuda_stream));
+  a.sync = (int32_t*)workspace;
+  a.part_ml = (float*)((uint8_t*)workspace + align_up(ATTN_SYNC_BYTES));
+  a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream))) return rc;
+  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }
@@ -950,8 +967,9 @@ int bita_tree_attention_static(const void* q, const void* k, const void* v, cons
   void* scratch = nullptr;
   rc = static_scratch_address(&scratch);
   if (rc) return rc;
-  // Every partial that the merge kernel reads is written by the slice kernel of the same call,
-  // so nothing in the shared array has to be cleared first.
+  // Every partial result that is read was written by the slices of the same call; the merge
+  // counters at the head of the array must be zero at launch and are cleared by the callee, in
+  // stream order, on every call.
   return bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
                              scratch, need, cuda_stream);
 }
