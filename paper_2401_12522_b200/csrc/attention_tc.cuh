@@ -142,7 +142,6 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
   constexpr int KS_P = ATT_KEYS / 16;        // k-steps of P.V
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_launch();
-  pdl_wait();
   const int h = blockIdx.x, s = blockIdx.y;
   const int b = blockIdx.z / a.row_tiles, rt = blockIdx.z - b * a.row_tiles;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -169,14 +168,7 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
   const bf16* pk = has_prompt ? a.prompt_k + (size_t)kvh * a.P * D : nullptr;
   const bf16* pv = has_prompt ? a.prompt_v + (size_t)kvh * a.P * D : nullptr;
 
-  // ---- stage Q rows, visibility words and prompt flags
-  for (int i = threadIdx.x; i < rows_cta * CH; i += nthreads) {
-    const int r = i / CH, c = i - r * CH;
-    const int gr = row0 + r;
-    const bool valid = gr < a.M;
-    const bf16* src = a.q + (((size_t)b * a.M + (valid ? gr : 0)) * a.H + h) * D + c * 8;
-    cp_async16(smem_u32(q_s) + swz<D>(r, c), src, valid);
-  }
+  // ---- stage visibility words and prompt flags (fixed by the tree template)
   for (int i = threadIdx.x; i < rows_cta * a.W; i += nthreads) {
     const int r = i / a.W, w = i - r * a.W;
     const int gr = row0 + r;
@@ -204,7 +196,30 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
     }
   };
 
-  if (c_begin < c_end) load_chunk(c_begin, 0);
+  // What does not depend on the kernel before this one is requested before waiting for it: the
+  // context slots [0, C) were written by earlier passes and the prompt prefix is a weight, so a
+  // chunk without block rows can be on its way while the projection that writes q and the block's
+  // own k, v is still finishing.  Up to two chunks (both buffers) are requested ahead.
+  auto early = [&](int ci) { return ci >= cache_chunks || (ci + 1) * ATT_KEYS <= C; };
+  int issued = c_begin;                                         // chunks below this index are requested
+  while (issued < c_end && issued < c_begin + 2 && early(issued)) {
+    load_chunk(issued, issued - c_begin);
+    cp_async_commit();
+    ++issued;
+  }
+  pdl_wait();
+  // ---- stage the Q rows
+  for (int i = threadIdx.x; i < rows_cta * CH; i += nthreads) {
+    const int r = i / CH, c = i - r * CH;
+    const int gr = row0 + r;
+    const bool valid = gr < a.M;
+    const bf16* src = a.q + (((size_t)b * a.M + (valid ? gr : 0)) * a.H + h) * D + c * 8;
+    cp_async16(smem_u32(q_s) + swz<D>(r, c), src, valid);
+  }
+  if (issued == c_begin && c_begin < c_end) {
+    load_chunk(c_begin, 0);
+    ++issued;
+  }
   cp_async_commit();
 
   float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
@@ -217,7 +232,7 @@ __global__ void __launch_bounds__(MAXW * 32, MAXW <= 5 ? 2 : 1) k_attn_tc(AttnAr
 
   for (int ci = c_begin; ci < c_end; ++ci) {
     const int buf = (ci - c_begin) & 1;
-    if (ci + 1 < c_end) load_chunk(ci + 1, buf ^ 1);
+    if (ci + 1 < c_end && ci + 1 >= issued) load_chunk(ci + 1, buf ^ 1);
     cp_async_commit();
     cp_async_wait<1>();
     __syncthreads();
