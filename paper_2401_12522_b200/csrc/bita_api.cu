@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "attention_tc.cuh"
+#include "attention_umma.cuh"
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "step_kernels.cuh"
@@ -341,9 +342,25 @@ void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
   *warps = w; *row_tiles = rt; *splits = s;
 }
 
+// Same for the tcgen05 engine: 128 query rows per CTA, one CTA per SM.
+void attn_shape_umma(int H, int B, int M, int* row_tiles, int* splits) {
+  const int rt = (M + AU_ROWS - 1) / AU_ROWS;
+  const int ctas = H * B * rt;
+  int s = 148 / ctas;
+  if (s < 1) s = 1;
+  if (s > 8) s = 8;
+  *row_tiles = rt; *splits = s;
+}
+
+bool attn_use_umma() {
+  static const bool on = getenv("BITA_ATTN_MMA_SYNC") == nullptr;
+  return on;
+}
+
 int attn_splits(int H, int B, int M) {
   int w, rt, s;
-  attn_shape(H, B, M, &w, &rt, &s);
+  if (attn_use_umma()) attn_shape_umma(H, B, M, &rt, &s);
+  else attn_shape(H, B, M, &w, &rt, &s);
   return s;
 }
 
@@ -376,7 +393,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.sel_val = (float*)take(R * BITA_MAX_TOPK * 4);
   t.pos = (int32_t*)take(R * 4);
   t.row_token = (int32_t*)take(R * 4);
-  const size_t S = 6;                        // upper bound of attn_splits
+  const size_t S = 8;                        // upper bound of attn_splits
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
@@ -472,7 +489,33 @@ GemmTcParams epi_store(float* out, int ldo) {
 
 // Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches the slices (and the
 // merge kernel where the slices cannot merge themselves).
+int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched) {
+  attn_shape_umma(a.H, a.B, a.M, &a.row_tiles, &a.S);
+  a.warps = 0;
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
+  const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
+  const size_t smem = 5 * tile + 2 * AU_ATOM + 1024;           // Q, 2 x (K, V), P
+  static bool attr_set = false;
+  if (!attr_set) {
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    attr_set = true;
+  }
+  // Slices merge inside the kernel when all CTAs of the launch fit one wave (one CTA per SM).
+  const int ctas = a.H * a.B * a.row_tiles;
+  if (a.S == 1 || ctas * a.S > 148 || ctas > ATTN_SYNC_SLOTS) a.sync = nullptr;
+  const bool merge_after = a.S > 1 && !a.sync;
+  if (n_launched) *n_launched = merge_after ? 2 : 1;
+  dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
+  int rc = a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<128>, a)
+                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<64>, a);
+  if (rc || !merge_after) return rc;
+  return a.D == 128 ? launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a)
+                    : launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
+}
+
 int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched) {
+  if (attn_use_umma()) return launch_attention_umma(a, pdl, s, n_launched);
   attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const int rows_cta = a.warps * 16;
