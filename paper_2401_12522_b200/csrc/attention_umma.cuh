@@ -241,6 +241,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
         return (visw[jj >> 5] >> (jj & 31)) & 1u;
       };
       if (ok) ok = mbar_wait(smem_u32(&bar_s_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
+      ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
       const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(i & 1) * AU_KEYS;
       // pass 1: row maximum over the visible keys
@@ -257,6 +258,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       const float corr = exp2f(m_run - sub);                    // 0 while nothing was seen before
       // P overwrites the tile the previous P V product reads, and the rescale touches its accumulator
       if (i > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(i - 1) & 1u, status);
+      ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       // pass 2: P = exp2(s * scale - max), row sum, bf16 tile
       float sum = 0.f;
@@ -281,8 +283,9 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       }
       tc_fence_before();
       mbar_arrive_cta(smem_u32(&bar_s_free[i & 1]));            // this S buffer may be overwritten
-      if (i > 0 && corr != 1.0f) {
-        // the maximum moved: bring this row of the accumulator to the new reference
+      if (i > 0 && __any_sync(0xffffffffu, corr != 1.0f)) {
+        // the maximum of some row of this warp moved: bring the accumulator rows to their new
+        // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch)
         for (int c0 = 0; c0 < D; c0 += 16) {
           float v[16];
           tmem_ld16(lane_addr + COL_O + (uint32_t)c0, v);
@@ -299,6 +302,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       mbar_arrive_cta(smem_u32(&bar_p_full));
     }
     if (n > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(n - 1) & 1u, status);
+    ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     pdl_wait();
     // ---- result of this slice: row r of O
