@@ -42,17 +42,58 @@ __device__ __forceinline__ uint64_t umma_smem_desc_mn(uint32_t addr, uint32_t lb
   return d;
 }
 
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+// 128 consecutive columns of this thread's TMEM lane, one wait for all of them.
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, float* v) {
+  uint32_t r[128];
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-      "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-      "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-      "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
-      "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%128];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%129];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%64, %65, %66, %67, %68, %69, %70, %71, %72, %73, %74, %75, %76, %77, %78, %79, %80, %81, %82, %83, %84, %85, %86, %87, %88, %89, %90, %91, %92, %93, %94, %95}, [%130];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%96, %97, %98, %99, %100, %101, %102, %103, %104, %105, %106, %107, %108, %109, %110, %111, %112, %113, %114, %115, %116, %117, %118, %119, %120, %121, %122, %123, %124, %125, %126, %127}, [%131];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95]), "=r"(r[96]), "=r"(r[97]), "=r"(r[98]), "=r"(r[99]), "=r"(r[100]), "=r"(r[101]), "=r"(r[102]), "=r"(r[103]), "=r"(r[104]), "=r"(r[105]), "=r"(r[106]), "=r"(r[107]), "=r"(r[108]), "=r"(r[109]), "=r"(r[110]), "=r"(r[111]), "=r"(r[112]), "=r"(r[113]), "=r"(r[114]), "=r"(r[115]), "=r"(r[116]), "=r"(r[117]), "=r"(r[118]), "=r"(r[119]), "=r"(r[120]), "=r"(r[121]), "=r"(r[122]), "=r"(r[123]), "=r"(r[124]), "=r"(r[125]), "=r"(r[126]), "=r"(r[127])
+      : "r"(taddr + 0u), "r"(taddr + 32u), "r"(taddr + 64u), "r"(taddr + 96u)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 128; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// 64 consecutive columns of this thread's TMEM lane, one wait for all of them.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
+  uint32_t r[64];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr + 0u), "r"(taddr + 32u)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_st128(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35};\n\t"
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%1], {%36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64, %65, %66, %67};\n\t"
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%2], {%68, %69, %70, %71, %72, %73, %74, %75, %76, %77, %78, %79, %80, %81, %82, %83, %84, %85, %86, %87, %88, %89, %90, %91, %92, %93, %94, %95, %96, %97, %98, %99};\n\t"
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%3], {%100, %101, %102, %103, %104, %105, %106, %107, %108, %109, %110, %111, %112, %113, %114, %115, %116, %117, %118, %119, %120, %121, %122, %123, %124, %125, %126, %127, %128, %129, %130, %131};\n\t"
+      "tcgen05.wait::st.sync.aligned;"
+      :
+      : "r"(taddr + 0u), "r"(taddr + 32u), "r"(taddr + 64u), "r"(taddr + 96u), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])), "r"(__float_as_uint(v[32])), "r"(__float_as_uint(v[33])), "r"(__float_as_uint(v[34])), "r"(__float_as_uint(v[35])), "r"(__float_as_uint(v[36])), "r"(__float_as_uint(v[37])), "r"(__float_as_uint(v[38])), "r"(__float_as_uint(v[39])), "r"(__float_as_uint(v[40])), "r"(__float_as_uint(v[41])), "r"(__float_as_uint(v[42])), "r"(__float_as_uint(v[43])), "r"(__float_as_uint(v[44])), "r"(__float_as_uint(v[45])), "r"(__float_as_uint(v[46])), "r"(__float_as_uint(v[47])), "r"(__float_as_uint(v[48])), "r"(__float_as_uint(v[49])), "r"(__float_as_uint(v[50])), "r"(__float_as_uint(v[51])), "r"(__float_as_uint(v[52])), "r"(__float_as_uint(v[53])), "r"(__float_as_uint(v[54])), "r"(__float_as_uint(v[55])), "r"(__float_as_uint(v[56])), "r"(__float_as_uint(v[57])), "r"(__float_as_uint(v[58])), "r"(__float_as_uint(v[59])), "r"(__float_as_uint(v[60])), "r"(__float_as_uint(v[61])), "r"(__float_as_uint(v[62])), "r"(__float_as_uint(v[63])), "r"(__float_as_uint(v[64])), "r"(__float_as_uint(v[65])), "r"(__float_as_uint(v[66])), "r"(__float_as_uint(v[67])), "r"(__float_as_uint(v[68])), "r"(__float_as_uint(v[69])), "r"(__float_as_uint(v[70])), "r"(__float_as_uint(v[71])), "r"(__float_as_uint(v[72])), "r"(__float_as_uint(v[73])), "r"(__float_as_uint(v[74])), "r"(__float_as_uint(v[75])), "r"(__float_as_uint(v[76])), "r"(__float_as_uint(v[77])), "r"(__float_as_uint(v[78])), "r"(__float_as_uint(v[79])), "r"(__float_as_uint(v[80])), "r"(__float_as_uint(v[81])), "r"(__float_as_uint(v[82])), "r"(__float_as_uint(v[83])), "r"(__float_as_uint(v[84])), "r"(__float_as_uint(v[85])), "r"(__float_as_uint(v[86])), "r"(__float_as_uint(v[87])), "r"(__float_as_uint(v[88])), "r"(__float_as_uint(v[89])), "r"(__float_as_uint(v[90])), "r"(__float_as_uint(v[91])), "r"(__float_as_uint(v[92])), "r"(__float_as_uint(v[93])), "r"(__float_as_uint(v[94])), "r"(__float_as_uint(v[95])), "r"(__float_as_uint(v[96])), "r"(__float_as_uint(v[97])), "r"(__float_as_uint(v[98])), "r"(__float_as_uint(v[99])), "r"(__float_as_uint(v[100])), "r"(__float_as_uint(v[101])), "r"(__float_as_uint(v[102])), "r"(__float_as_uint(v[103])), "r"(__float_as_uint(v[104])), "r"(__float_as_uint(v[105])), "r"(__float_as_uint(v[106])), "r"(__float_as_uint(v[107])), "r"(__float_as_uint(v[108])), "r"(__float_as_uint(v[109])), "r"(__float_as_uint(v[110])), "r"(__float_as_uint(v[111])), "r"(__float_as_uint(v[112])), "r"(__float_as_uint(v[113])), "r"(__float_as_uint(v[114])), "r"(__float_as_uint(v[115])), "r"(__float_as_uint(v[116])), "r"(__float_as_uint(v[117])), "r"(__float_as_uint(v[118])), "r"(__float_as_uint(v[119])), "r"(__float_as_uint(v[120])), "r"(__float_as_uint(v[121])), "r"(__float_as_uint(v[122])), "r"(__float_as_uint(v[123])), "r"(__float_as_uint(v[124])), "r"(__float_as_uint(v[125])), "r"(__float_as_uint(v[126])), "r"(__float_as_uint(v[127]))
       : "memory");
 }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_st64(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33};\n\t"
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%1], {%34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64, %65};\n\t"
+      "tcgen05.wait::st.sync.aligned;"
+      :
+      : "r"(taddr + 0u), "r"(taddr + 32u), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])), "r"(__float_as_uint(v[32])), "r"(__float_as_uint(v[33])), "r"(__float_as_uint(v[34])), "r"(__float_as_uint(v[35])), "r"(__float_as_uint(v[36])), "r"(__float_as_uint(v[37])), "r"(__float_as_uint(v[38])), "r"(__float_as_uint(v[39])), "r"(__float_as_uint(v[40])), "r"(__float_as_uint(v[41])), "r"(__float_as_uint(v[42])), "r"(__float_as_uint(v[43])), "r"(__float_as_uint(v[44])), "r"(__float_as_uint(v[45])), "r"(__float_as_uint(v[46])), "r"(__float_as_uint(v[47])), "r"(__float_as_uint(v[48])), "r"(__float_as_uint(v[49])), "r"(__float_as_uint(v[50])), "r"(__float_as_uint(v[51])), "r"(__float_as_uint(v[52])), "r"(__float_as_uint(v[53])), "r"(__float_as_uint(v[54])), "r"(__float_as_uint(v[55])), "r"(__float_as_uint(v[56])), "r"(__float_as_uint(v[57])), "r"(__float_as_uint(v[58])), "r"(__float_as_uint(v[59])), "r"(__float_as_uint(v[60])), "r"(__float_as_uint(v[61])), "r"(__float_as_uint(v[62])), "r"(__float_as_uint(v[63]))
+      : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -244,14 +285,21 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
       const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(i & 1) * AU_KEYS;
-      // pass 1: row maximum over the visible keys
+      // the whole row of scores into registers (one TMEM round trip); the buffer is free again
+      float sv[AU_KEYS];
+      tmem_ld128(s_addr, sv);
+      tc_fence_before();
+      mbar_arrive_cta(smem_u32(&bar_s_free[i & 1]));
       float mx = -INFINITY;
-      for (int c0 = 0; c0 < AU_KEYS; c0 += 16) {
-        float v[16];
-        tmem_ld16(s_addr + (uint32_t)c0, v);
+      if (all_vis) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (all_vis || visible(c0 + j)) mx = fmaxf(mx, v[j]);
+        for (int j = 0; j < AU_KEYS; ++j) mx = fmaxf(mx, sv[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < AU_KEYS; ++j) {
+          if (!visible(j)) sv[j] = -INFINITY;                   // exp2(-inf) = 0 below
+          mx = fmaxf(mx, sv[j]);
+        }
       }
       const float m_new = fmaxf(m_run, mx * sc);
       const float sub = m_new == -INFINITY ? 0.f : m_new;
@@ -260,40 +308,29 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       if (i > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(i - 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
-      // pass 2: P = exp2(s * scale - max), row sum, bf16 tile
+      // P = exp2(s * scale - max), row sum, bf16 tile
       float sum = 0.f;
-      for (int c0 = 0; c0 < AU_KEYS; c0 += 16) {
-        float v[16];
-        tmem_ld16(s_addr + (uint32_t)c0, v);
-        uint32_t pk[8];
 #pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-          const float p0 = (all_vis || visible(c0 + j)) ? exp2f(v[j] * sc - sub) : 0.f;
-          const float p1 = (all_vis || visible(c0 + j + 1)) ? exp2f(v[j + 1] * sc - sub) : 0.f;
+      for (int c0 = 0; c0 < AU_KEYS; c0 += 8) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+          const float p0 = exp2f(sv[c0 + j] * sc - sub), p1 = exp2f(sv[c0 + j + 1] * sc - sub);
           sum += p0 + p1;
           pk[j >> 1] = pack_bf16x2(p0, p1);
         }
-        const int cc = c0 >> 3;                                 // 16-byte chunk index of keys c0 .. c0+7
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, cc)), "r"(pk[0]), "r"(pk[1]),
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, c0 >> 3)), "r"(pk[0]), "r"(pk[1]),
                      "r"(pk[2]), "r"(pk[3])
                      : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, cc + 1)), "r"(pk[4]), "r"(pk[5]),
-                     "r"(pk[6]), "r"(pk[7])
-                     : "memory");
       }
-      tc_fence_before();
-      mbar_arrive_cta(smem_u32(&bar_s_free[i & 1]));            // this S buffer may be overwritten
       if (i > 0 && __any_sync(0xffffffffu, corr != 1.0f)) {
         // the maximum of some row of this warp moved: bring the accumulator rows to their new
         // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch)
-        for (int c0 = 0; c0 < D; c0 += 16) {
-          float v[16];
-          tmem_ld16(lane_addr + COL_O + (uint32_t)c0, v);
+        float ov[D];
+        if constexpr (D == 128) tmem_ld128(lane_addr + COL_O, ov); else tmem_ld64(lane_addr + COL_O, ov);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] *= corr;
-          tmem_st16(lane_addr + COL_O + (uint32_t)c0, v);
-        }
-        tmem_wait_st();
+        for (int j = 0; j < D; ++j) ov[j] *= corr;
+        if constexpr (D == 128) tmem_st128(lane_addr + COL_O, ov); else tmem_st64(lane_addr + COL_O, ov);
       }
       l_run = l_run * corr + sum;
       m_run = m_new;
@@ -306,25 +343,23 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
     tc_fence_after();
     pdl_wait();
     // ---- result of this slice: row r of O
+    float ov[D];
+    if (n > 0 && ok) {
+      if constexpr (D == 128) tmem_ld128(lane_addr + COL_O, ov); else tmem_ld64(lane_addr + COL_O, ov);
+    } else {
+#pragma unroll
+      for (int j = 0; j < D; ++j) ov[j] = 0.f;
+    }
     if (a.S == 1) {
       const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-      bf16* dst = a.out + (((size_t)b * a.M + (row_live ? gr : 0)) * a.H + h) * D;
-      for (int c0 = 0; c0 < D; c0 += 16) {
-        float v[16];
-        if (n > 0 && ok) {
-          tmem_ld16(lane_addr + COL_O + (uint32_t)c0, v);
-        } else {
+      if (row_live) {
+        bf16* dst = a.out + (((size_t)b * a.M + gr) * a.H + h) * D;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0.f;
-        }
-        if (row_live) {
-          uint4 w0, w1;
-          w0.x = pack_bf16x2(v[0] * inv, v[1] * inv);   w0.y = pack_bf16x2(v[2] * inv, v[3] * inv);
-          w0.z = pack_bf16x2(v[4] * inv, v[5] * inv);   w0.w = pack_bf16x2(v[6] * inv, v[7] * inv);
-          w1.x = pack_bf16x2(v[8] * inv, v[9] * inv);   w1.y = pack_bf16x2(v[10] * inv, v[11] * inv);
-          w1.z = pack_bf16x2(v[12] * inv, v[13] * inv); w1.w = pack_bf16x2(v[14] * inv, v[15] * inv);
-          *reinterpret_cast<uint4*>(dst + c0) = w0;
-          *reinterpret_cast<uint4*>(dst + c0 + 8) = w1;
+        for (int c0 = 0; c0 < D; c0 += 8) {
+          uint4 w;
+          w.x = pack_bf16x2(ov[c0] * inv, ov[c0 + 1] * inv);     w.y = pack_bf16x2(ov[c0 + 2] * inv, ov[c0 + 3] * inv);
+          w.z = pack_bf16x2(ov[c0 + 4] * inv, ov[c0 + 5] * inv); w.w = pack_bf16x2(ov[c0 + 6] * inv, ov[c0 + 7] * inv);
+          *reinterpret_cast<uint4*>(dst + c0) = w;
         }
       }
     } else {
@@ -332,21 +367,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       if (row_live) {
         a.part_ml[(pbase + gr) * 2] = m_run;
         a.part_ml[(pbase + gr) * 2 + 1] = l_run;
-      }
-      float* dst = a.part_acc + (pbase + (row_live ? gr : 0)) * D;
-      for (int c0 = 0; c0 < D; c0 += 16) {
-        float v[16];
-        if (n > 0 && ok) {
-          tmem_ld16(lane_addr + COL_O + (uint32_t)c0, v);
-        } else {
+        float* dst = a.part_acc + (pbase + gr) * D;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0.f;
-        }
-        if (row_live) {
-#pragma unroll
-          for (int j = 0; j < 16; j += 4)
-            *reinterpret_cast<float4*>(dst + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-        }
+        for (int j = 0; j < D; j += 4)
+          *reinterpret_cast<float4*>(dst + j) = make_float4(ov[j], ov[j + 1], ov[j + 2], ov[j + 3]);
       }
       __threadfence();
     }
