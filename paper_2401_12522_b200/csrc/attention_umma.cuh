@@ -15,7 +15,8 @@
 //                  lies in the cache ([key][D], i.e. MN-major for this product): the same staging
 //                  layout serves K (K-major for Q K^T) and V (MN-major for P V).
 // Roles: warps 0-3 softmax (TMEM lane group = warp), warp 4 issues the MMAs (one lane), warp 5
-// stages Q and the K/V chunks with cp.async (two chunk buffers).  Everything is handed over
+// brings Q and the K/V chunks in with TMA (two chunk buffers; box = 64 features x 128 rows, 128-byte
+// swizzle, no multicast) and clears the V rows past the last key before handing a chunk over.  Everything is handed over
 // through mbarriers with bounded waits; a wait that runs out raises the status word, the kernel
 // drains and frees its TMEM.
 #pragma once
@@ -99,19 +100,34 @@ __device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// 3-D tiled TMA load global -> shared (no multicast), completion on an mbarrier.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+
+// Tensor maps of one attention call.  q: (D, H, B*M) box (64, 1, 128); k, v: (D, C_max, B*H_kv) box
+// (64, 128, 1); prompt_k, prompt_v: (D, P, H_kv) box (64, 128, 1) (copies of k, v when there is no prefix).
+struct AttnMaps {
+  CUtensorMap q, k, v, pk, pv;
+};
+
 // Byte offset of element (row r, 16-byte chunk c) in a tile staged as 64-element-wide swizzle atoms.
 __device__ __forceinline__ uint32_t au_off(int r, int c) {
   return (uint32_t)((c >> 3) * AU_ATOM + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
 template <int D>
-__global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
+__global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_constant__ AttnMaps maps, AttnArgs a) {
   constexpr int CH = D / 8;                         // 16-byte chunks per row
   constexpr int TILE = (D / 64) * AU_ATOM;          // bytes of a staged [128][D] tile
   constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;
   constexpr uint32_t TMEM_COLS = 512;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2], bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done;
+  __shared__ __align__(8) uint64_t bar_tma[2], bar_q;
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
 
@@ -130,7 +146,9 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
       mbar_init(smem_u32(&bar_kv_empty[i]), 1);
       mbar_init(smem_u32(&bar_s_full[i]), 1);
       mbar_init(smem_u32(&bar_s_free[i]), 128);
+      mbar_init(smem_u32(&bar_tma[i]), 1);
     }
+    mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_p_full), 128);
     mbar_init(smem_u32(&bar_pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -159,57 +177,79 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
 
   if (warp == 5) {
     // ---------------- loader: Q once, then K/V chunks into the two chunk buffers
-    const bf16* kb = a.k + ((size_t)b * a.H_kv + kvh) * (size_t)a.C_max * D;
-    const bf16* vb = a.v + ((size_t)b * a.H_kv + kvh) * (size_t)a.C_max * D;
-    const bf16* pk = has_prompt ? a.prompt_k + (size_t)kvh * a.P * D : nullptr;
-    const bf16* pv = has_prompt ? a.prompt_v + (size_t)kvh * a.P * D : nullptr;
-    auto load_chunk = [&](int i) {
+    const uint32_t chunk_bytes = 2u * TILE;
+    auto issue_chunk = [&](int i) {                              // lane 0 only
       const int ci = c_begin + i;
       const uint32_t ks = kv_s + (uint32_t)(i & 1) * 2 * TILE, vs = ks + TILE;
       const bool is_prompt = ci >= cache_chunks;
-      const int key0 = is_prompt ? 0 : ci * AU_KEYS;
-      const int limit = is_prompt ? a.P : n_cache;
-      const bf16* ksrc = is_prompt ? pk : kb;
-      const bf16* vsrc = is_prompt ? pv : vb;
-      for (int j = lane; j < AU_KEYS * CH; j += 32) {
-        const int r = j / CH, c = j - r * CH;
-        const bool valid = key0 + r < limit;
-        const size_t off = (size_t)(valid ? key0 + r : 0) * D + c * 8;
-        cp_async16(ks + au_off(r, c), ksrc + off, valid);
-        cp_async16(vs + au_off(r, c), vsrc + off, valid);
+      const uint32_t bar = smem_u32(&bar_tma[i & 1]);
+      mbar_expect_tx(bar, chunk_bytes);
+#pragma unroll
+      for (int hf = 0; hf < D / 64; ++hf) {
+        if (is_prompt) {
+          tma_load_3d(ks + hf * AU_ATOM, &maps.pk, hf * 64, 0, kvh, bar);
+          tma_load_3d(vs + hf * AU_ATOM, &maps.pv, hf * 64, 0, kvh, bar);
+        } else {
+          tma_load_3d(ks + hf * AU_ATOM, &maps.k, hf * 64, ci * AU_KEYS, b * a.H_kv + kvh, bar);
+          tma_load_3d(vs + hf * AU_ATOM, &maps.v, hf * 64, ci * AU_KEYS, b * a.H_kv + kvh, bar);
+        }
       }
     };
     // chunks without block rows depend on nothing the previous kernel writes
     auto early = [&](int i) { const int ci = c_begin + i; return ci >= cache_chunks || (ci + 1) * AU_KEYS <= C; };
     int issued = 0;
-    while (issued < n && issued < 2 && early(issued)) { load_chunk(issued); ++issued; }
-    pdl_wait();
-    for (int j = lane; j < AU_ROWS * CH; j += 32) {
-      const int r = j / CH, c = j - r * CH;
-      const int gr = row0 + r;
-      const bool valid = gr < a.M;
-      const bf16* src = a.q + (((size_t)b * a.M + (valid ? gr : 0)) * a.H + h) * D + c * 8;
-      cp_async16(q_s + au_off(r, c), src, valid);
+    while (issued < n && issued < 2 && early(issued)) {
+      if (lane == 0) issue_chunk(issued);
+      ++issued;
     }
-    if (issued == 0 && n > 0) { load_chunk(0); issued = 1; }
-    cp_async_commit();
-    cp_async_wait<0>();
-    fence_async_smem();
-    __syncwarp();
-    if (lane == 0) {
-      for (int i = 0; i < issued; ++i) mbar_arrive_cta(smem_u32(&bar_kv_full[i]));
+    pdl_wait();
+    if (lane == 0 && n > 0) {
+      mbar_expect_tx(smem_u32(&bar_q), (uint32_t)TILE);
+#pragma unroll
+      for (int hf = 0; hf < D / 64; ++hf)
+        tma_load_3d(q_s + hf * AU_ATOM, &maps.q, hf * 64, h, b * a.M + row0, smem_u32(&bar_q));
     }
     bool ok = true;
-    for (int i = issued; i < n && ok; ++i) {
-      // the buffer was last used by chunk i - 2: free once its P V product has completed
-      ok = mbar_wait(smem_u32(&bar_kv_empty[i & 1]), ((uint32_t)(i >> 1) & 1u) ^ 1u, status);
+    for (int i = 0; i < n && ok; ++i) {
+      if (i >= issued) {
+        // the buffer was last used by chunk i - 2: free once its P V product has completed
+        if (i >= 2) ok = mbar_wait(smem_u32(&bar_kv_empty[i & 1]), ((uint32_t)(i >> 1) & 1u) ^ 1u, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) issue_chunk(i);
+        issued = i + 1;
+      }
+      ok = mbar_wait(smem_u32(&bar_tma[i & 1]), (uint32_t)(i >> 1) & 1u, status);
+      ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      load_chunk(i);
-      cp_async_commit();
-      cp_async_wait<0>();
-      fence_async_smem();
+      // V rows past the last key of the cache may hold anything (a stale or never written slot):
+      // they meet P = 0, but 0 x NaN is NaN, so they are cleared.  (Rows past the end of the
+      // tensor, and of the prompt prefix, arrive as zeros.)
+      const int ci = c_begin + i;
+      if (ci < cache_chunks) {
+        const int live_rows = n_cache - ci * AU_KEYS;
+        if (live_rows < AU_KEYS) {
+          const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
+          for (int j = lane; j < (AU_KEYS - live_rows) * CH; j += 32) {
+            const int r = live_rows + j / CH, c = j % CH;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + au_off(r, c)), "r"(0u) : "memory");
+          }
+          fence_async_smem();
+        }
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive_cta(smem_u32(&bar_kv_full[i & 1]));
+      // the next chunk's buffer frees when the product before this one is done: ask for it now
+      if (i + 1 < n && i + 1 >= issued) {
+        if (i + 1 >= 2) ok = mbar_wait(smem_u32(&bar_kv_empty[(i + 1) & 1]), ((uint32_t)((i + 1) >> 1) & 1u) ^ 1u, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) issue_chunk(i + 1);
+        issued = i + 2;
+      }
+    }
+    if (!ok) {
+      for (int i = 0; i < 64; ++i) __nanosleep(1000);            // let the copies in flight land
     }
   } else if (warp == 4) {
     // ---------------- MMA issuer
@@ -228,7 +268,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(AttnArgs a) {
         }
         umma_commit(smem_u32(&bar_s_full[i & 1]));
       };
-      ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, status);
+      ok = mbar_wait(smem_u32(&bar_q), 0, status);
+      if (ok) ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, status);
       tc_fence_after();
       if (ok) issue_s(0);
       for (int i = 0; i < n && ok; ++i) {

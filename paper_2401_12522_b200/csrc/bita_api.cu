@@ -252,6 +252,23 @@ int make_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows) {
   return BITA_OK;
 }
 
+// bf16 tensor [d2][d1][d0] (d0 contiguous, the given byte strides) -> 3-D map, 128-byte swizzle, zero fill.
+int make_map3(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1,
+              uint64_t stride2, uint32_t box1, uint32_t box2) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return BITA_ERR_CUDA;
+  if (((uintptr_t)base & 15) || (stride1 & 15) || (stride2 & 15)) return BITA_ERR_INVALID_ARG;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1, stride2};
+  cuuint32_t box[3] = {64, box1, box2};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return BITA_ERR_CUDA; }
+  return BITA_OK;
+}
+
 // One weight matrix (or a gate/up pair) as the projection kernel sees it.
 struct GemmDesc {
   CUtensorMap a0, a1;
@@ -429,6 +446,7 @@ struct bita_ctx {
   std::vector<GemmDesc> d_qkv, d_o, d_gu, d_dn;
   GemmDesc d_head;
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
+  std::map<std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>, AttnMaps> attn_map_cache;
   bool pdl;                             // programmatic dependent launch between the kernels of a pass
 
   // optional per-family event timing
@@ -489,8 +507,38 @@ GemmTcParams epi_store(float* out, int ldo) {
 
 // Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches the slices (and the
 // merge kernel where the slices cannot merge themselves).
-int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched) {
+// Tensor maps of an attention call; `cache` (may be null) keeps them across calls with the same
+// buffers and shapes.
+using AttnMapKey = std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>;
+int attn_maps(const AttnArgs& a, std::map<AttnMapKey, AttnMaps>* cache, AttnMaps* out) {
+  const AttnMapKey key{a.q, a.k, a.v, a.prompt_k, a.B * a.M, a.H * 1024 + a.H_kv, a.C_max, a.P * 1024 + a.D};
+  if (cache) {
+    auto it = cache->find(key);
+    if (it != cache->end()) { *out = it->second; return BITA_OK; }
+  }
+  const uint64_t D = a.D, row = D * 2;
+  int rc;
+  if ((rc = make_map3(&out->q, a.q, D, a.H, (uint64_t)a.B * a.M, row, row * a.H, 1, AU_ROWS))) return rc;
+  if ((rc = make_map3(&out->k, a.k, D, a.C_max, (uint64_t)a.B * a.H_kv, row, row * a.C_max, AU_KEYS, 1))) return rc;
+  if ((rc = make_map3(&out->v, a.v, D, a.C_max, (uint64_t)a.B * a.H_kv, row, row * a.C_max, AU_KEYS, 1))) return rc;
+  if (a.P > 0 && a.prompt_k && a.prompt_v) {
+    if ((rc = make_map3(&out->pk, a.prompt_k, D, a.P, a.H_kv, row, row * a.P, AU_KEYS, 1))) return rc;
+    if ((rc = make_map3(&out->pv, a.prompt_v, D, a.P, a.H_kv, row, row * a.P, AU_KEYS, 1))) return rc;
+  } else {
+    out->pk = out->k;
+    out->pv = out->v;
+  }
+  if (cache) cache->emplace(key, *out);
+  return BITA_OK;
+}
+
+int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
   attn_shape_umma(a.H, a.B, a.M, &a.row_tiles, &a.S);
+  AttnMaps maps;
+  {
+    int rc = attn_maps(a, cache, &maps);
+    if (rc) return rc;
+  }
   a.warps = 0;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
@@ -507,15 +555,15 @@ int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched)
   const bool merge_after = a.S > 1 && !a.sync;
   if (n_launched) *n_launched = merge_after ? 2 : 1;
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
-  int rc = a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<128>, a)
-                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<64>, a);
+  int rc = a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<128>, maps, a)
+                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<64>, maps, a);
   if (rc || !merge_after) return rc;
   return a.D == 128 ? launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a)
                     : launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
 
-int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched) {
-  if (attn_use_umma()) return launch_attention_umma(a, pdl, s, n_launched);
+int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
+  if (attn_use_umma()) return launch_attention_umma(a, pdl, s, n_launched, cache);
   attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const int rows_cta = a.warps * 16;
@@ -613,7 +661,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     {
       Timed t(c, 1);
       int n = 0;
-      if ((rc = launch_attention(a, pdl, s, &n))) return rc;
+      if ((rc = launch_attention(a, pdl, s, &n, &c->attn_map_cache))) return rc;
       c->launches += n;
     }
     if ((rc = single(op_o(l)))) return rc;
@@ -967,7 +1015,7 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   a.part_ml = (float*)((uint8_t*)workspace + align_up(ATTN_SYNC_BYTES));
   a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr))) return rc;
+  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }
