@@ -114,6 +114,12 @@ struct AttnMaps {
   CUtensorMap q, k, v, pk, pv;
 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // Byte offset of element (row r, 16-byte chunk c) in a tile staged as 64-element-wide swizzle atoms.
 __device__ __forceinline__ uint32_t au_off(int r, int c) {
   return (uint32_t)((c >> 3) * AU_ATOM + r * 128 + (((c & 7) ^ (r & 7)) << 4));
@@ -126,8 +132,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;
   constexpr uint32_t TMEM_COLS = 512;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2], bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done;
-  __shared__ __align__(8) uint64_t bar_tma[2], bar_q;
+  // K and V tiles of a chunk buffer are handed over separately: a K tile is free again once its
+  // Q K^T chain is done (long before the chunk's P V product), so the next K is on its way early.
+  __shared__ __align__(8) uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
+  __shared__ __align__(8) uint64_t bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done, bar_q, bar_vfix;
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
 
@@ -142,13 +150,15 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bar_kv_full[i]), 1);
-      mbar_init(smem_u32(&bar_kv_empty[i]), 1);
+      mbar_init(smem_u32(&bar_k_full[i]), 1);
+      mbar_init(smem_u32(&bar_k_empty[i]), 1);
+      mbar_init(smem_u32(&bar_v_full[i]), 1);
+      mbar_init(smem_u32(&bar_v_empty[i]), 1);
       mbar_init(smem_u32(&bar_s_full[i]), 1);
       mbar_init(smem_u32(&bar_s_free[i]), 128);
-      mbar_init(smem_u32(&bar_tma[i]), 1);
     }
     mbar_init(smem_u32(&bar_q), 1);
+    mbar_init(smem_u32(&bar_vfix), 1);
     mbar_init(smem_u32(&bar_p_full), 128);
     mbar_init(smem_u32(&bar_pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -174,34 +184,32 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   const int n_chunks = cache_chunks + (has_prompt ? 1 : 0);
   const int c_begin = (int)((long)n_chunks * s / a.S), c_end = (int)((long)n_chunks * (s + 1) / a.S);
   const int n = c_end - c_begin;
+  // The cache chunk that holds the last key may end in slots that were never written: their V rows
+  // are cleared before the P V product (`fix` = index of that chunk within this slice, or -1).
+  const int fix = (n_cache % AU_KEYS != 0 && cache_chunks - 1 >= c_begin && cache_chunks - 1 < c_end)
+                      ? cache_chunks - 1 - c_begin : -1;
 
   if (warp == 5) {
-    // ---------------- loader: Q once, then K/V chunks into the two chunk buffers
-    const uint32_t chunk_bytes = 2u * TILE;
-    auto issue_chunk = [&](int i) {                              // lane 0 only
+    // ---------------- loader (one lane issues; the warp clears the rows of the `fix` chunk)
+    auto issue_tile = [&](int i, bool v_tile) {                  // lane 0 only
       const int ci = c_begin + i;
-      const uint32_t ks = kv_s + (uint32_t)(i & 1) * 2 * TILE, vs = ks + TILE;
+      const uint32_t dst = kv_s + (uint32_t)(i & 1) * 2 * TILE + (v_tile ? TILE : 0);
       const bool is_prompt = ci >= cache_chunks;
-      const uint32_t bar = smem_u32(&bar_tma[i & 1]);
-      mbar_expect_tx(bar, chunk_bytes);
+      const uint32_t bar = smem_u32(v_tile ? &bar_v_full[i & 1] : &bar_k_full[i & 1]);
+      const CUtensorMap* map = is_prompt ? (v_tile ? &maps.pv : &maps.pk) : (v_tile ? &maps.v : &maps.k);
+      mbar_expect_tx(bar, (uint32_t)TILE);
 #pragma unroll
-      for (int hf = 0; hf < D / 64; ++hf) {
-        if (is_prompt) {
-          tma_load_3d(ks + hf * AU_ATOM, &maps.pk, hf * 64, 0, kvh, bar);
-          tma_load_3d(vs + hf * AU_ATOM, &maps.pv, hf * 64, 0, kvh, bar);
-        } else {
-          tma_load_3d(ks + hf * AU_ATOM, &maps.k, hf * 64, ci * AU_KEYS, b * a.H_kv + kvh, bar);
-          tma_load_3d(vs + hf * AU_ATOM, &maps.v, hf * 64, ci * AU_KEYS, b * a.H_kv + kvh, bar);
-        }
-      }
+      for (int hf = 0; hf < D / 64; ++hf)
+        tma_load_3d(dst + hf * AU_ATOM, map, hf * 64, is_prompt ? 0 : ci * AU_KEYS, is_prompt ? kvh : b * a.H_kv + kvh, bar);
     };
     // chunks without block rows depend on nothing the previous kernel writes
     auto early = [&](int i) { const int ci = c_begin + i; return ci >= cache_chunks || (ci + 1) * AU_KEYS <= C; };
-    int issued = 0;
-    while (issued < n && issued < 2 && early(issued)) {
-      if (lane == 0) issue_chunk(issued);
-      ++issued;
+    int k_issued = 0, v_issued = 0;
+    while (k_issued < n && k_issued < 2 && early(k_issued)) {
+      if (lane == 0) { issue_tile(k_issued, false); issue_tile(k_issued, true); }
+      ++k_issued;
     }
+    v_issued = k_issued;
     pdl_wait();
     if (lane == 0 && n > 0) {
       mbar_expect_tx(smem_u32(&bar_q), (uint32_t)TILE);
@@ -210,42 +218,40 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         tma_load_3d(q_s + hf * AU_ATOM, &maps.q, hf * 64, h, b * a.M + row0, smem_u32(&bar_q));
     }
     bool ok = true;
-    for (int i = 0; i < n && ok; ++i) {
-      if (i >= issued) {
-        // the buffer was last used by chunk i - 2: free once its P V product has completed
-        if (i >= 2) ok = mbar_wait(smem_u32(&bar_kv_empty[i & 1]), ((uint32_t)(i >> 1) & 1u) ^ 1u, status);
+    if (k_issued == 0 && n > 0) {
+      if (lane == 0) issue_tile(0, false);
+      k_issued = 1;
+    }
+    // The MMA thread runs S(0), S(1), PV(0), S(2), PV(1), ...: K(j+1) waits for S(j-1), then V(j)
+    // waits for PV(j-2), in that order.
+    for (int j = 0; j < n && ok; ++j) {
+      if (j + 1 < n && j + 1 >= k_issued) {
+        if (j + 1 >= 2) ok = mbar_wait(smem_u32(&bar_k_empty[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        if (lane == 0) issue_chunk(i);
-        issued = i + 1;
+        if (lane == 0) issue_tile(j + 1, false);
+        k_issued = j + 2;
       }
-      ok = mbar_wait(smem_u32(&bar_tma[i & 1]), (uint32_t)(i >> 1) & 1u, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      // V rows past the last key of the cache may hold anything (a stale or never written slot):
-      // they meet P = 0, but 0 x NaN is NaN, so they are cleared.  (Rows past the end of the
-      // tensor, and of the prompt prefix, arrive as zeros.)
-      const int ci = c_begin + i;
-      if (ci < cache_chunks) {
-        const int live_rows = n_cache - ci * AU_KEYS;
-        if (live_rows < AU_KEYS) {
-          const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
-          for (int j = lane; j < (AU_KEYS - live_rows) * CH; j += 32) {
-            const int r = live_rows + j / CH, c = j % CH;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + au_off(r, c)), "r"(0u) : "memory");
-          }
-          fence_async_smem();
+      if (j >= v_issued) {
+        if (j >= 2) ok = mbar_wait(smem_u32(&bar_v_empty[j & 1]), ((uint32_t)(j >> 1) & 1u) ^ 1u, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) issue_tile(j, true);
+        v_issued = j + 1;
+      }
+      if (j == fix) {
+        ok = mbar_wait(smem_u32(&bar_v_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const int live_rows = n_cache - (c_begin + j) * AU_KEYS;
+        const uint32_t vs = kv_s + (uint32_t)(j & 1) * 2 * TILE + TILE;
+        for (int t = lane; t < (AU_KEYS - live_rows) * CH; t += 32) {
+          const int r = live_rows + t / CH, c = t % CH;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + au_off(r, c)), "r"(0u) : "memory");
         }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cta(smem_u32(&bar_kv_full[i & 1]));
-      // the next chunk's buffer frees when the product before this one is done: ask for it now
-      if (i + 1 < n && i + 1 >= issued) {
-        if (i + 1 >= 2) ok = mbar_wait(smem_u32(&bar_kv_empty[(i + 1) & 1]), ((uint32_t)((i + 1) >> 1) & 1u) ^ 1u, status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane == 0) issue_chunk(i + 1);
-        issued = i + 2;
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cta(smem_u32(&bar_vfix));
       }
     }
     if (!ok) {
@@ -267,14 +273,15 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           umma_bf16(d_tmem, da, db, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(smem_u32(&bar_s_full[i & 1]));
+        umma_commit(smem_u32(&bar_k_empty[i & 1]));
       };
       ok = mbar_wait(smem_u32(&bar_q), 0, status);
-      if (ok) ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, status);
+      if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, status);
       tc_fence_after();
       if (ok) issue_s(0);
       for (int i = 0; i < n && ok; ++i) {
         if (i + 1 < n) {                                                  // S of the next chunk while this one is in softmax
-          ok = mbar_wait(smem_u32(&bar_kv_full[(i + 1) & 1]), (uint32_t)((i + 1) >> 1) & 1u, status);
+          ok = mbar_wait(smem_u32(&bar_k_full[(i + 1) & 1]), (uint32_t)((i + 1) >> 1) & 1u, status);
           if (ok && i + 1 >= 2)
             ok = mbar_wait(smem_u32(&bar_s_free[(i + 1) & 1]), ((uint32_t)((i + 1) >> 1) & 1u) ^ 1u, status);
           if (!ok) break;
@@ -282,6 +289,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           issue_s(i + 1);
         }
         ok = mbar_wait(smem_u32(&bar_p_full), (uint32_t)i & 1u, status);
+        if (ok) ok = mbar_wait(smem_u32(&bar_v_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
+        if (ok && i == fix) ok = mbar_wait(smem_u32(&bar_vfix), 0, status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
@@ -291,7 +300,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           const uint64_t db = umma_smem_desc_mn(vs + kk * 16 * 128, AU_ATOM);
           umma_bf16(tmem + COL_O, da, db, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bar_kv_empty[i & 1]));
+        umma_commit(smem_u32(&bar_v_empty[i & 1]));
         umma_commit(smem_u32(&bar_pv_done));
       }
     }
@@ -356,7 +365,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         uint32_t pk[4];
 #pragma unroll
         for (int j = 0; j < 8; j += 2) {
-          const float p0 = exp2f(sv[c0 + j] * sc - sub), p1 = exp2f(sv[c0 + j + 1] * sc - sub);
+          const float p0 = ex2_approx(sv[c0 + j] * sc - sub), p1 = ex2_approx(sv[c0 + j + 1] * sc - sub);
           sum += p0 + p1;
           pk[j >> 1] = pack_bf16x2(p0, p1);
         }
