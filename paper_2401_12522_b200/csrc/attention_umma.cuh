@@ -312,8 +312,11 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     const float sc = a.scale_log2;
     uint32_t visw[8];
 #pragma unroll
-    for (int w = 0; w < 8; ++w)
+    for (int w = 0; w < 8; ++w) {
       visw[w] = (row_live && w < a.W) ? a.vis[(size_t)b * a.vis_batch_stride + (size_t)gr * a.W + w] : 0u;
+      const int nb = a.M - 32 * w;                              // block rows this word can name
+      if (nb < 32) visw[w] &= nb <= 0 ? 0u : ((1u << nb) - 1u);
+    }
     const bool sees_p = has_prompt && row_live && a.sees_prompt[(size_t)b * a.sp_batch_stride + gr] != 0;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     float m_run = -INFINITY, l_run = 0.f;
@@ -323,14 +326,39 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       const bool is_prompt = ci >= cache_chunks;
       const int key0 = is_prompt ? 0 : ci * AU_KEYS;
       const bool all_vis = !is_prompt && key0 + AU_KEYS <= C && row_live;
-      auto visible = [&](int j) -> bool {                       // key j of the chunk for this row
-        if (is_prompt) return sees_p && j < a.P;
-        const int key = key0 + j;
-        if (key < C) return row_live;
-        if (key >= n_cache) return false;
-        const int jj = key - C;
-        return (visw[jj >> 5] >> (jj & 31)) & 1u;
-      };
+      // Visibility of the chunk's 128 keys for this row as four 32-bit words: context keys are
+      // seen by every live row, block keys according to the row's ancestor bitmask (shifted to the
+      // key's place), prompt keys by mask rows only; keys past the last one by nobody.
+      uint32_t vm[4] = {0u, 0u, 0u, 0u};
+      if (row_live && !all_vis) {
+        if (is_prompt) {
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const int nb = a.P - 32 * w;                        // prompt keys in this word
+            vm[w] = !sees_p || nb <= 0 ? 0u : (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u));
+          }
+        } else {
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const int j0 = key0 + 32 * w - C;                   // block row index of the word's first key
+            uint32_t word;
+            if (j0 <= -32) {
+              word = 0xffffffffu;                               // all context
+            } else {
+              // bits [j0, j0 + 32) of the row's bitmask (bits below 0 are context: ones)
+              const int q = j0 >= 0 ? j0 >> 5 : -1, sh = j0 & 31;
+              uint32_t lo = q < 0 ? 0xffffffffu : 0u, hi = 0u;
+#pragma unroll
+              for (int t = 0; t < 8; ++t) {
+                if (t == q) lo = visw[t];
+                if (t == q + 1) hi = visw[t];
+              }
+              word = sh == 0 ? lo : __funnelshift_r(lo, hi, sh);
+            }
+            vm[w] = word;
+          }
+        }
+      }
       if (ok) ok = mbar_wait(smem_u32(&bar_s_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
@@ -347,7 +375,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       } else {
 #pragma unroll
         for (int j = 0; j < AU_KEYS; ++j) {
-          if (!visible(j)) sv[j] = -INFINITY;                   // exp2(-inf) = 0 below
+          if (!((vm[j >> 5] >> (j & 31)) & 1u)) sv[j] = -INFINITY;   // exp2(-inf) = 0 below
           mx = fmaxf(mx, sv[j]);
         }
       }
