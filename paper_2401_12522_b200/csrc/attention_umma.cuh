@@ -1,8 +1,8 @@
 // Tree-based attention (Sec. 3.2, Fig. 6) on the tcgen05 tensor cores.
 //
-// Same interface, key enumeration, slicing and partial-result format as attention_tc.cuh; what
-// differs is the inner engine.  One CTA = one query head x one key slice x up to 128 query rows.
-// Keys are walked in chunks of 128:
+// One CTA = one query head x one key slice x up to 128 query rows (arguments, slicing and the
+// partial-result format: attention_common.cuh).  The slice's keys are walked in chunks of 128; the
+// cache chunks come first, the prompt-prefix chunk last:
 //   S = Q K^T      one UMMA chain, M = 128 (query rows), N = 128 (keys), K = D; Q and the K chunk
 //                  sit in shared memory as K-major 128-byte-swizzled tiles; S lands in TMEM with
 //                  lane = query row, column = key (two S buffers alternate);
@@ -21,7 +21,7 @@
 // drains and frees its TMEM.
 #pragma once
 
-#include "attention_tc.cuh"
+#include "attention_common.cuh"
 #include "gemm_tc.cuh"
 
 namespace bita {
@@ -454,7 +454,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
   }
 
-  // ---- merge inside the kernel (all slices resident), as in attention_tc.cuh
+  // ---- merge inside the kernel: all slices of this (sequence, head, row tile) are resident CTAs,
+  // none of which waits before its partial results are out, so the wait ends; bounded all the same.
   tc_fence_before();
   __syncthreads();
   if (a.S > 1 && a.sync) {
@@ -478,7 +479,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     __syncthreads();
     const int rows_here = min(AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
-    for (int r = r_lo + warp; r < r_hi; r += AU_THREADS / 32) attn_merge_row<D>(a, b, h, row0 + r, lane);
+    attn_merge_rows<D>(a, b, h, row0, r_lo, r_hi, warp, AU_THREADS / 32, lane);
     __syncthreads();
     if (threadIdx.x == 0) {
       const int old = atomicAdd(departed, 1);

@@ -10,7 +10,6 @@
 #include <tuple>
 #include <vector>
 
-#include "attention_tc.cuh"
 #include "attention_umma.cuh"
 #include "common.cuh"
 #include "gemm_tc.cuh"
@@ -347,20 +346,8 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
 
-// Attention launch shape: warps per CTA, row tiles, key slices (about two CTAs per SM in total).
-void attn_shape(int H, int B, int M, int* warps, int* row_tiles, int* splits) {
-  const int groups = (M + 15) / 16;            // 16-row groups, one warp each
-  const int rt = (groups + 7) / 8;             // at most 8 warps per CTA
-  const int w = (groups + rt - 1) / rt;        // spread evenly over the row tiles
-  const int ctas = H * B * rt;
-  int s = 296 / ctas;                          // every slice resident at once (two CTAs per SM)
-  if (s < 1) s = 1;
-  if (s > 6) s = 6;
-  *warps = w; *row_tiles = rt; *splits = s;
-}
-
-// Same for the tcgen05 engine: 128 query rows per CTA, one CTA per SM.
-void attn_shape_umma(int H, int B, int M, int* row_tiles, int* splits) {
+// Attention launch shape: row tiles of 128 query rows and key slices, one CTA per SM in total.
+void attn_shape(int H, int B, int M, int* row_tiles, int* splits) {
   const int rt = (M + AU_ROWS - 1) / AU_ROWS;
   const int ctas = H * B * rt;
   int s = 148 / ctas;
@@ -369,15 +356,9 @@ void attn_shape_umma(int H, int B, int M, int* row_tiles, int* splits) {
   *row_tiles = rt; *splits = s;
 }
 
-bool attn_use_umma() {
-  static const bool on = getenv("BITA_ATTN_MMA_SYNC") == nullptr;
-  return on;
-}
-
 int attn_splits(int H, int B, int M) {
-  int w, rt, s;
-  if (attn_use_umma()) attn_shape_umma(H, B, M, &rt, &s);
-  else attn_shape(H, B, M, &w, &rt, &s);
+  int rt, s;
+  attn_shape(H, B, M, &rt, &s);
   return s;
 }
 
@@ -504,9 +485,6 @@ GemmTcParams epi_store(float* out, int ldo) {
   return p;
 }
 
-
-// Fills the launch-shape fields of `a` (warps, row_tiles, S, scale) and launches the slices (and the
-// merge kernel where the slices cannot merge themselves).
 // Tensor maps of an attention call; `cache` (may be null) keeps them across calls with the same
 // buffers and shapes.
 using AttnMapKey = std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>;
@@ -532,14 +510,15 @@ int attn_maps(const AttnArgs& a, std::map<AttnMapKey, AttnMaps>* cache, AttnMaps
   return BITA_OK;
 }
 
-int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
-  attn_shape_umma(a.H, a.B, a.M, &a.row_tiles, &a.S);
+// Fills the launch-shape fields of `a` (row_tiles, S, scale) and launches the slices (and the merge
+// kernel where the slices cannot merge themselves).
+int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
+  attn_shape(a.H, a.B, a.M, &a.row_tiles, &a.S);
   AttnMaps maps;
   {
     int rc = attn_maps(a, cache, &maps);
     if (rc) return rc;
   }
-  a.warps = 0;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
   const size_t smem = 5 * tile + 2 * AU_ATOM + 1024;           // Q, 2 x (K, V), P
@@ -560,42 +539,6 @@ int launch_attention_umma(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched,
   if (rc || !merge_after) return rc;
   return a.D == 128 ? launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a)
                     : launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
-}
-
-int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
-  if (attn_use_umma()) return launch_attention_umma(a, pdl, s, n_launched, cache);
-  attn_shape(a.H, a.B, a.M, &a.warps, &a.row_tiles, &a.S);
-  a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
-  const int rows_cta = a.warps * 16;
-  const size_t smem = (size_t)rows_cta * a.D * 2 + 4 * (size_t)ATT_KEYS * a.D * 2 + (size_t)rows_cta * a.W * 4 +
-                      rows_cta + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_tc<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
-    attr_set = true;
-  }
-  dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
-  const dim3 blk(a.warps * 32);
-  // The slices merge inside the kernel when they all run in one wave (two CTAs per SM for blocks of
-  // up to five warps, one otherwise); a single slice writes the output itself.
-  const int wave = a.warps <= 5 ? 296 : 148;
-  if (a.S == 1 || a.H * a.S * a.B * a.row_tiles > wave || a.B * a.H * a.row_tiles > ATTN_SYNC_SLOTS) a.sync = nullptr;
-  const bool merge_after = a.S > 1 && !a.sync;
-  if (n_launched) *n_launched = merge_after ? 2 : 1;
-  int rc;
-  if (a.D == 128) {
-    rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 5>, a)
-                      : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<128, 8>, a);
-    if (rc || !merge_after) return rc;
-    return launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a);
-  }
-  rc = a.warps <= 5 ? launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 5>, a)
-                    : launch(s, pdl, g1, blk, smem, 1, k_attn_tc<64, 8>, a);
-  if (rc || !merge_after) return rc;
-  return launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
 
 // The layer stack over one packed block, then (optionally) the LM head and selection.
