@@ -19,7 +19,7 @@ from helpers import block_for, oracle_model, orc, prompt_tokens, synth
 # tolerances of the parity target
 HIDDEN_REL_L2 = 1e-2          # error a layer adds, relative L2 over the whole block (see layer_increment)
 LOGIT_TOL_RMS = 3e-2          # max |delta| <= 3e-2 * RMS(oracle logits) ...
-LOGIT_TOL_PER_HIDDEN = 6.0    # ... or 6 x the accumulated hidden error where that is larger (see _compare_float)
+LOGIT_TOL_PER_HIDDEN = 6.0    # ... or 6 x the accumulated hidden error of the worst row where that is larger (see _compare_float)
 KV_REL_L2 = 1e-2              # cache contents are bf16 roundings of the oracle's fp64 values
 
 
@@ -72,7 +72,12 @@ class Lockstep:
                 ref = float(np.linalg.norm(o))
                 e = layer_increment(err_abs, prev, ref)
                 prev = err_abs
-                acc_rel = err_abs / (ref if ref > 0 else 1.0)
+                # A row of logits inherits the error of its own row of the hidden state, and the rows
+                # differ (mask rows sit further out than tree rows): the logits are bounded with the
+                # worst row, the per-layer criterion stays on the whole block.
+                row_ref = np.linalg.norm(o, axis=-1)
+                row_rel = np.linalg.norm(g - o, axis=-1) / np.where(row_ref > 0, row_ref, 1.0)
+                acc_rel = max(err_abs / (ref if ref > 0 else 1.0), float(row_rel.max()))
                 self.max_hidden = max(self.max_hidden, e)
                 self.max_hidden_acc = max(self.max_hidden_acc, acc_rel)
                 assert e <= HIDDEN_REL_L2, f"hidden layer {l}: adds rel L2 {e:.3e} (accumulated {acc_rel:.3e})"
