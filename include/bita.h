@@ -197,9 +197,11 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
  *   prompt_k/v  DEVICE bf16 [H_kv][P][D] or NULL; sees_prompt DEVICE uint8 [B][M] or NULL
  *   ctx_len     DEVICE int32 [B]: C per sequence, C + M <= C_max
  *   out    DEVICE bf16 [B][M][H*D]
- * `workspace` DEVICE scratch of bita_attention_workspace_bytes, 256-byte aligned; the call
- * clears the merge counters at its head (a stream-ordered memset) and overwrites the rest.
- * A wait between key slices that runs out (2 s) leaves wrong output rather than a hang. */
+ * `workspace` DEVICE scratch of bita_attention_workspace_bytes, 256-byte aligned: room for the
+ * partial results of the key slices.  (The slices normally run as one thread-block cluster and
+ * merge on chip; the scratch is written only when that launch form is refused and a second
+ * kernel has to merge.)  A wait between key slices that runs out (2 s) leaves wrong output
+ * rather than a hang. */
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes);
 int bita_tree_attention(const void* q, const void* k, const void* v, const uint32_t* vis,
                         const void* prompt_k, const void* prompt_v, const uint8_t* sees_prompt,
@@ -226,10 +228,9 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
  *     allocation).  Make that first call outside any stream capture.
  *   - The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
- *     That is harmless here: each call clears the merge counters at the head of the array (a
- *     stream-ordered memset, no allocation) and overwrites every other slot it later reads.  But
- *     two calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
- *     order them on one stream or with events.
+ *     That is harmless here, because each call overwrites every slot it later reads, but two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it: order
+ *     them on one stream or with events.
  * Results are the same as bita_tree_attention's. */
 #define BITA_STATIC_SCRATCH_BYTES (8u << 20)
 int bita_tree_attention_static(const void* q, const void* k, const void* v, const uint32_t* vis,

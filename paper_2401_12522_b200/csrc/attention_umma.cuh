@@ -18,7 +18,8 @@
 // brings Q and the K/V chunks in with TMA (two chunk buffers; box = 64 features x 128 rows, 128-byte
 // swizzle, no multicast) and clears the V rows past the last key before handing a chunk over.  Everything is handed over
 // through mbarriers with bounded waits; a wait that runs out raises the status word, the kernel
-// drains and frees its TMEM.
+// drains and frees its TMEM.  Several key slices of one (sequence, head, row tile) run as one
+// thread-block cluster and merge their partial results through distributed shared memory.
 #pragma once
 
 #include "attention_common.cuh"
@@ -62,6 +63,48 @@ struct AttnMaps {
   CUtensorMap q, k, v, pk, pv;
 };
 
+// ---- cluster helpers: a peer CTA's shared memory and mbarriers
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+// Bounded wait with cluster-scope acquire (the data were written by other CTAs of the cluster).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int32_t* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((i & 63u) == 63u) {
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > TC_WAIT_LIMIT_NS) break;
+    }
+  }
+  atomicExch(status, BITA_ERR_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t remote_addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote_addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_dsmem_f2(uint32_t remote_addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote_addr));
+  return v;
+}
+
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -79,11 +122,13 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   constexpr int TILE = (D / 64) * AU_ATOM;          // bytes of a staged [128][D] tile
   constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;
   constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t PSTRIDE = (D + 4) * 4;         // bytes of a partial row in shared memory: m, l, pad, O[D]
   extern __shared__ uint8_t smem_raw[];
   // K and V tiles of a chunk buffer are handed over separately: a K tile is free again once its
   // Q K^T chain is done (long before the chunk's P V product), so the next K is on its way early.
   __shared__ __align__(8) uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
   __shared__ __align__(8) uint64_t bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done, bar_q, bar_vfix;
+  __shared__ __align__(8) uint64_t bar_cl_in, bar_cl_out;      // cluster merge: partials in / reads done
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
 
@@ -107,6 +152,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
     mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_vfix), 1);
+    mbar_init(smem_u32(&bar_cl_in), (uint32_t)a.S);
+    mbar_init(smem_u32(&bar_cl_out), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_p_full), 128);
     mbar_init(smem_u32(&bar_pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -120,6 +167,11 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (a.S > 1 && a.cluster) {
+    // peers arrive on this CTA's merge barriers: they must be initialised cluster-wide first
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  }
   const uint32_t tmem = tmem_slot;
   int32_t* status = a.status ? a.status : &status_local;
   if (threadIdx.x == 0) pdl_launch();
@@ -388,6 +440,18 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           *reinterpret_cast<uint4*>(dst + c0) = w;
         }
       }
+    } else if (a.cluster) {
+      // partial result of this row into this CTA's shared memory (the chunk buffers are free:
+      // every copy into them has landed and every MMA that read them is complete)
+      if (row_live) {
+        const uint32_t prow = kv_s + (uint32_t)r * PSTRIDE;
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(prow), "f"(m_run), "f"(l_run) : "memory");
+#pragma unroll
+        for (int j = 0; j < D; j += 4)
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(prow + 16 + j * 4), "f"(ov[j]), "f"(ov[j + 1]),
+                       "f"(ov[j + 2]), "f"(ov[j + 3])
+                       : "memory");
+      }
     } else {
       const size_t pbase = (((size_t)b * a.H + h) * a.S + s) * a.M;
       if (row_live) {
@@ -402,37 +466,69 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
   }
 
-  // ---- merge inside the kernel: all slices of this (sequence, head, row tile) are resident CTAs,
-  // none of which waits before its partial results are out, so the wait ends; bounded all the same.
+  // ---- merge inside the cluster: the S slices of this (sequence, head, row tile) are the CTAs of
+  // one cluster (rank = slice).  Each leaves its partial rows in its own shared memory, tells every
+  // peer, and once all S are in merges an equal share of the rows, reading the peers' partials
+  // through distributed shared memory, in slice order.  A second round of arrivals keeps every CTA
+  // alive until its peers have finished reading it.  Both waits are bounded mbarrier waits.
   tc_fence_before();
   __syncthreads();
-  if (a.S > 1 && a.sync) {
-    const int n_sync = a.B * a.H * a.row_tiles;
-    int32_t* arrived = a.sync + ((size_t)b * a.H + h) * a.row_tiles + rt;
-    int32_t* departed = arrived + n_sync;
+  if (a.S > 1 && a.cluster) {
     if (threadIdx.x == 0) {
-      atomicAdd(arrived, 1);
-      unsigned long long w0 = 0;
-      bool ok = true;
-      for (uint32_t spin = 0; ld_acquire_gpu(arrived) < a.S; ++spin) {
-        if ((spin & 63u) == 63u) {
-          const unsigned long long now = global_ns();
-          if (w0 == 0) w0 = now;
-          else if (now - w0 > TC_WAIT_LIMIT_NS) { ok = false; break; }
-        }
-      }
-      if (!ok) atomicExch(status, BITA_ERR_TIMEOUT);
-      __threadfence();
+      asm volatile("fence.acq_rel.cluster;" ::: "memory");
+      for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_in), (uint32_t)p));
     }
-    __syncthreads();
+    mbar_wait_cluster(smem_u32(&bar_cl_in), 0, status);
+    constexpr int VW = D / 32;
     const int rows_here = min(AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
-    attn_merge_rows<D>(a, b, h, row0, r_lo, r_hi, warp, AU_THREADS / 32, lane);
+    for (int r = r_lo + warp; r < r_hi; r += AU_THREADS / 32) {
+      float ms[8], ls[8], v[8][VW];
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        ms[p] = -INFINITY;
+        ls[p] = 0.f;
+#pragma unroll
+        for (int e = 0; e < VW; ++e) v[p][e] = 0.f;
+        if (p < a.S) {
+          const uint32_t prow = mapa_u32(kv_s + (uint32_t)r * PSTRIDE, (uint32_t)p);
+          const float2 ml = ld_dsmem_f2(prow);
+          ms[p] = ml.x;
+          ls[p] = ml.y;
+          if constexpr (VW == 4) {
+            const float4 t = ld_dsmem_f4(prow + 16 + lane * 16);
+            v[p][0] = t.x; v[p][1] = t.y; v[p][2] = t.z; v[p][3] = t.w;
+          } else {
+            const float2 t = ld_dsmem_f2(prow + 16 + lane * 8);
+            v[p][0] = t.x; v[p][1] = t.y;
+          }
+        }
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) mx = fmaxf(mx, ms[p]);
+      float l = 0.f, o[VW];
+#pragma unroll
+      for (int e = 0; e < VW; ++e) o[e] = 0.f;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        if (ms[p] == -INFINITY) continue;
+        const float w = exp2f(ms[p] - mx);
+        l += ls[p] * w;
+#pragma unroll
+        for (int e = 0; e < VW; ++e) o[e] += v[p][e] * w;
+      }
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
+      bf16* dst = a.out + (((size_t)b * a.M + row0 + r) * a.H + h) * D + lane * VW;
+#pragma unroll
+      for (int e = 0; e < VW; e += 2)
+        *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
-      const int old = atomicAdd(departed, 1);
-      if (old == a.S - 1) { *arrived = 0; *departed = 0; }
+      for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_out), (uint32_t)p));
     }
+    mbar_wait_cluster(smem_u32(&bar_cl_out), 0, status);
   }
   if (warp == 4) {
     tc_fence_after();

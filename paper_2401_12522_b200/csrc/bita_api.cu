@@ -278,8 +278,6 @@ struct GemmDesc {
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
-constexpr int ATTN_SYNC_SLOTS = 2048;   // (sequence, head, row tile) triples with counters for the in-kernel merge
-constexpr size_t ATTN_SYNC_BYTES = 2 * ATTN_SYNC_SLOTS * 4;
 constexpr int GEMM_MAX_CTAS = 296;
 constexpr int GEMM_MAX_SPLITS = 8;
 
@@ -346,13 +344,18 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
 
-// Attention launch shape: row tiles of 128 query rows and key slices, one CTA per SM in total.
+// Attention launch shape: row tiles of 128 query rows, and key slices.  The slices of a (sequence,
+// head, row tile) form a thread-block cluster; the slice count is the largest cluster size whose
+// clusters all fit the GPU at once (one CTA per SM; concurrent clusters seen on a B200: 74 of size
+// 2, 45 of 3, 33 of 4, 22 of 6, 15 of 8).  More clusters than that would still be correct (they
+// run in waves), just not faster.
 void attn_shape(int H, int B, int M, int* row_tiles, int* splits) {
   const int rt = (M + AU_ROWS - 1) / AU_ROWS;
-  const int ctas = H * B * rt;
-  int s = 148 / ctas;
-  if (s < 1) s = 1;
-  if (s > 8) s = 8;
+  const int groups = H * B * rt;
+  static const int size[5] = {8, 6, 4, 3, 2}, fit[5] = {15, 22, 33, 45, 74};
+  int s = 1;
+  for (int i = 0; i < 5; ++i)
+    if (groups <= fit[i]) { s = size[i]; break; }
   *row_tiles = rt; *splits = s;
 }
 
@@ -365,7 +368,7 @@ int attn_splits(int H, int B, int M) {
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
-  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt; int32_t* attn_sync;
+  int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
 };
@@ -396,7 +399,6 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
   t.gemm_cnt = (int32_t*)take(4096 * 4);
-  t.attn_sync = (int32_t*)take(ATTN_SYNC_BYTES);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -528,15 +530,22 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_set = true;
   }
-  // Slices merge inside the kernel when all CTAs of the launch fit one wave (one CTA per SM).
-  const int ctas = a.H * a.B * a.row_tiles;
-  if (a.S == 1 || ctas * a.S > 148 || ctas > ATTN_SYNC_SLOTS) a.sync = nullptr;
-  const bool merge_after = a.S > 1 && !a.sync;
-  if (n_launched) *n_launched = merge_after ? 2 : 1;
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
-  int rc = a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<128>, maps, a)
-                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, 1, k_attn_umma<64>, maps, a);
-  if (rc || !merge_after) return rc;
+  auto run = [&](unsigned cluster_y) {
+    return a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<128>, maps, a)
+                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<64>, maps, a);
+  };
+  if (n_launched) *n_launched = 1;
+  if (a.S == 1) return run(1);
+  a.cluster = 1;
+  int rc = run((unsigned)a.S);
+  if (rc == BITA_OK) return rc;
+  // The cluster launch was refused: the slices leave their partial results in global memory
+  // and a second kernel merges them.
+  (void)cudaGetLastError();
+  a.cluster = 0;
+  if (n_launched) *n_launched = 2;
+  if ((rc = run(1))) return rc;
   return a.D == 128 ? launch(s, pdl, g2, dim3(64), 0, 1, k_attn_merge<128>, a)
                     : launch(s, pdl, g2, dim3(32), 0, 1, k_attn_merge<64>, a);
 }
@@ -600,7 +609,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
-    a.sync = b.attn_sync; a.status = &b.state->status;
+    a.status = &b.state->status;
     {
       Timed t(c, 1);
       int n = 0;
@@ -737,7 +746,6 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
   if (cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
-  if (cudaMemsetAsync(c->b.attn_sync, 0, ATTN_SYNC_BYTES, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
@@ -932,7 +940,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
   if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
   const size_t S = attn_splits(H, B, M);
-  *out_bytes = align_up(ATTN_SYNC_BYTES) + align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
+  *out_bytes = align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
   return BITA_OK;
 }
 
@@ -952,10 +960,8 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
   a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
-  // workspace: merge counters (zero at launch: cleared here, in stream order), then the partial results
-  CU_TRY(cudaMemsetAsync(workspace, 0, ATTN_SYNC_BYTES, (cudaStream_t)cuda_stream));
-  a.sync = (int32_t*)workspace;
-  a.part_ml = (float*)((uint8_t*)workspace + align_up(ATTN_SYNC_BYTES));
+  // workspace: partial results of the key slices (used when the slices cannot run as a cluster)
+  a.part_ml = (float*)workspace;
   a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
   if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr))) return rc;
@@ -1001,9 +1007,8 @@ int bita_tree_attention_static(const void* q, const void* k, const void* v, cons
   void* scratch = nullptr;
   rc = static_scratch_address(&scratch);
   if (rc) return rc;
-  // Every partial result that is read was written by the slices of the same call; the merge
-  // counters at the head of the array must be zero at launch and are cleared by the callee, in
-  // stream order, on every call.
+  // Every partial result that the merge reads was written by the slices of the same call, so
+  // nothing in the shared array has to be cleared first.
   return bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
                              scratch, need, cuda_stream);
 }
