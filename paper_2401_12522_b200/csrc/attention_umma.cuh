@@ -182,7 +182,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   const int cache_chunks = (n_cache + AU_KEYS - 1) / AU_KEYS;
   const bool has_prompt = a.P > 0 && a.prompt_k && a.prompt_v && a.sees_prompt;
   const int n_chunks = cache_chunks + (has_prompt ? 1 : 0);
-  const int c_begin = (int)((long)n_chunks * s / a.S), c_end = (int)((long)n_chunks * (s + 1) / a.S);
+  // Slice boundaries rounded up: the surplus chunks go to the first slices, so the last ones, which
+  // hold the block's own keys (not available before the dependency wait), have the least to do.
+  const int c_begin = (int)(((long)n_chunks * s + a.S - 1) / a.S);
+  const int c_end = (int)(((long)n_chunks * (s + 1) + a.S - 1) / a.S);
   const int n = c_end - c_begin;
   // The cache chunk that holds the last key may end in slots that were never written: their V rows
   // are cleared before the P V product (`fix` = index of that chunk within this slice, or -1).
@@ -482,47 +485,57 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     constexpr int VW = D / 32;
     const int rows_here = min(AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
-    for (int r = r_lo + warp; r < r_hi; r += AU_THREADS / 32) {
-      float ms[8], ls[8], v[8][VW];
+    constexpr int NW = AU_THREADS / 32, RR = 3;                 // rows per warp whose loads fly together
+    for (int r0 = r_lo + warp; r0 < r_hi; r0 += NW * RR) {
+      float ms[RR][8], ls[RR][8], v[RR][8][VW];
 #pragma unroll
-      for (int p = 0; p < 8; ++p) {
-        ms[p] = -INFINITY;
-        ls[p] = 0.f;
+      for (int u = 0; u < RR; ++u) {
+        const int r = min(r0 + u * NW, r_hi - 1);               // clamped: surplus slots redo the last row
 #pragma unroll
-        for (int e = 0; e < VW; ++e) v[p][e] = 0.f;
-        if (p < a.S) {
-          const uint32_t prow = mapa_u32(kv_s + (uint32_t)r * PSTRIDE, (uint32_t)p);
-          const float2 ml = ld_dsmem_f2(prow);
-          ms[p] = ml.x;
-          ls[p] = ml.y;
-          if constexpr (VW == 4) {
-            const float4 t = ld_dsmem_f4(prow + 16 + lane * 16);
-            v[p][0] = t.x; v[p][1] = t.y; v[p][2] = t.z; v[p][3] = t.w;
-          } else {
-            const float2 t = ld_dsmem_f2(prow + 16 + lane * 8);
-            v[p][0] = t.x; v[p][1] = t.y;
+        for (int p = 0; p < 8; ++p) {
+          ms[u][p] = -INFINITY;
+          ls[u][p] = 0.f;
+#pragma unroll
+          for (int e = 0; e < VW; ++e) v[u][p][e] = 0.f;
+          if (p < a.S) {
+            const uint32_t prow = mapa_u32(kv_s + (uint32_t)r * PSTRIDE, (uint32_t)p);
+            const float2 ml = ld_dsmem_f2(prow);
+            ms[u][p] = ml.x;
+            ls[u][p] = ml.y;
+            if constexpr (VW == 4) {
+              const float4 t = ld_dsmem_f4(prow + 16 + lane * 16);
+              v[u][p][0] = t.x; v[u][p][1] = t.y; v[u][p][2] = t.z; v[u][p][3] = t.w;
+            } else {
+              const float2 t = ld_dsmem_f2(prow + 16 + lane * 8);
+              v[u][p][0] = t.x; v[u][p][1] = t.y;
+            }
           }
         }
       }
-      float mx = -INFINITY;
 #pragma unroll
-      for (int p = 0; p < 8; ++p) mx = fmaxf(mx, ms[p]);
-      float l = 0.f, o[VW];
+      for (int u = 0; u < RR; ++u) {
+        const int r = r0 + u * NW;
+        if (r >= r_hi) break;
+        float mx = -INFINITY;
 #pragma unroll
-      for (int e = 0; e < VW; ++e) o[e] = 0.f;
+        for (int p = 0; p < 8; ++p) mx = fmaxf(mx, ms[u][p]);
+        float l = 0.f, o[VW];
 #pragma unroll
-      for (int p = 0; p < 8; ++p) {
-        if (ms[p] == -INFINITY) continue;
-        const float w = exp2f(ms[p] - mx);
-        l += ls[p] * w;
+        for (int e = 0; e < VW; ++e) o[e] = 0.f;
 #pragma unroll
-        for (int e = 0; e < VW; ++e) o[e] += v[p][e] * w;
+        for (int p = 0; p < 8; ++p) {
+          if (ms[u][p] == -INFINITY) continue;
+          const float w = exp2f(ms[u][p] - mx);
+          l += ls[u][p] * w;
+#pragma unroll
+          for (int e = 0; e < VW; ++e) o[e] += v[u][p][e] * w;
+        }
+        const float inv = l > 0.f ? 1.0f / l : 0.f;
+        bf16* dst = a.out + (((size_t)b * a.M + row0 + r) * a.H + h) * D + lane * VW;
+#pragma unroll
+        for (int e = 0; e < VW; e += 2)
+          *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
       }
-      const float inv = l > 0.f ? 1.0f / l : 0.f;
-      bf16* dst = a.out + (((size_t)b * a.M + row0 + r) * a.H + h) * D + lane * VW;
-#pragma unroll
-      for (int e = 0; e < VW; e += 2)
-        *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
