@@ -474,50 +474,34 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
     __syncthreads();
     // Sum rows t0 .. t0+cnt of the partial tiles into `stg` (local row order), in split order.  A
-    // thread takes 16-byte items; sixteen loads fly together: four items x four splits, or (more
-    // than four splits: fewer rows per split, so fewer items) two items x eight splits.
+    // thread takes 16-byte items; the loads of four items (four splits each) fly together.
     const int items = cnt * (TC_BLOCK_N / 4);
     const float4* src = reinterpret_cast<const float4*>(part_tile) + (size_t)t0 * (TC_BLOCK_N / 4);
     const int stride4 = (int)(tile_elems / 4);               // between the splits' tiles
-    if (p.splits <= 4) {
-      for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
+    for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
+      float4 a4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) a4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int r0 = 0; r0 < p.splits; r0 += 4) {
         float4 v[4][4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int i = min(i0 + u * TC_THREADS, items - 1);
 #pragma unroll
           for (int r = 0; r < 4; ++r)
-            if (r < p.splits) v[u][r] = __ldcg(src + (size_t)r * stride4 + i);
+            if (r0 + r < p.splits) v[u][r] = __ldcg(src + (size_t)(r0 + r) * stride4 + i);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
           for (int r = 0; r < 4; ++r)
-            if (r < p.splits) { a4.x += v[u][r].x; a4.y += v[u][r].y; a4.z += v[u][r].z; a4.w += v[u][r].w; }
-          const int i = i0 + u * TC_THREADS;
-          if (i < items) reinterpret_cast<float4*>(stg)[i] = a4;
+            if (r0 + r < p.splits) { a4[u].x += v[u][r].x; a4[u].y += v[u][r].y; a4[u].z += v[u][r].z; a4[u].w += v[u][r].w; }
         }
       }
-    } else {
-      for (int i0 = threadIdx.x; i0 < items; i0 += 2 * TC_THREADS) {
-        float4 v[2][8];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int i = min(i0 + u * TC_THREADS, items - 1);
-#pragma unroll
-          for (int r = 0; r < 8; ++r)
-            if (r < p.splits) v[u][r] = __ldcg(src + (size_t)r * stride4 + i);
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-          for (int r = 0; r < 8; ++r)
-            if (r < p.splits) { a4.x += v[u][r].x; a4.y += v[u][r].y; a4.z += v[u][r].z; a4.w += v[u][r].w; }
-          const int i = i0 + u * TC_THREADS;
-          if (i < items) reinterpret_cast<float4*>(stg)[i] = a4;
-        }
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * TC_THREADS;
+        if (i < items) reinterpret_cast<float4*>(stg)[i] = a4[u];
       }
     }
     __syncthreads();
