@@ -421,6 +421,63 @@ def run_attn_sweep():
                 del q, k, v, flush
 
 
+def run_next_rows(args, shape):
+    """Measurements beyond the headline step: the first pass (Algorithm 1, t = 1) as a timed path, and
+    the cost side of the template comparison (Sec. 4.3): step latency per tree template at this
+    model shape.  One JSON line each; device-resident, CUDA events, no planted acceptance."""
+    from paper_2401_12522_b200 import Bita
+    from paper_2401_12522_b200.build import build
+    build()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    peak, _ = _peaks()
+    weights = synth.make_weights(shape, MODEL_SEED, dtype=torch.bfloat16, device=dev)
+    prompt = synth.uniform_ints(replica_plan(0, shape)["prompt_seed"], 5001, shape.prompt_len, shape.V).tolist()
+    n, steps = shape.n_mask, 24
+    templates = [
+        ("straightforward (chain of top-1 drafts, one group)", synth.chain_template(n)),
+        ("product-rule tree of the configuration, one group", synth.product_rule_template(shape.tree_K, shape.tree_B)),
+        ("efficient comb tree k=5, a group per node (paper default)", synth.comb_template(n, 5)),
+        ("efficient comb tree k=3, a group per node", synth.comb_template(n, 3)),
+    ]
+    for name, tmpl in templates:
+        rows = 1 + tmpl.N + tmpl.G * n
+        depth = max(tmpl.depths(), default=0)
+        C_max = shape.prompt_len + (steps + 8) * (depth + 1) + rows + 64
+        ctx = Bita(shape, weights, tmpl, C_max=C_max, device=dev)
+        ctx.reset()
+        # ---- first pass: chunks of 128 rows through the same kernels, then the first tree
+        times = []
+        for it in range(3):
+            ctx.reset()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.prefill(prompt)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        pre_ms = min(times)
+        flops = 2.0 * shape.streamed_params * shape.prompt_len
+        # ---- steps with the model's own drafts (random-init masks: acceptance ~ 0, so this is cost only)
+        for s in range(4):
+            ctx.step_enqueue(None)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(steps):
+            ctx.step_enqueue(None)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx.step_finish()
+        ms = e0.elapsed_time(e1) / steps
+        print(json.dumps({"metric": "step_latency_by_template", "workload": shape.name, "template": name,
+                          "nodes": tmpl.N, "groups": tmpl.G, "rows": rows, "ms_per_step": ms,
+                          "weights_gb_per_s": shape.streamed_params * 2 / ms / 1e6,
+                          "hbm_frac": shape.streamed_params * 2 / ms / 1e6 / peak,
+                          "prefill": {"tokens": shape.prompt_len, "ms": pre_ms, "tokens_per_s": shape.prompt_len / pre_ms * 1e3,
+                                      "tflops": flops / pre_ms / 1e9}}))
+        ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -433,9 +490,15 @@ def main():
     ap.add_argument("--cpu-samples", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--attn-sweep", action="store_true", help="time the tree-attention kernel alone over the sweep shapes")
+    ap.add_argument("--next-rows", action="store_true",
+                    help="first pass as a timed path and step latency per tree template (one JSON line per template)")
     args = ap.parse_args()
     if args.attn_sweep:
         run_attn_sweep()
+        return
+    if args.next_rows:
+        shape = synth.CONFIGS[args.workload]
+        run_next_rows(args, shape.with_layers(args.layers) if args.layers else shape)
         return
     if args.warmup < 3:
         args.warmup = 3
