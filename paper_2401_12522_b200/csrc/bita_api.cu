@@ -327,10 +327,11 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
   const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  // Small blocks run two CTAs per SM (half the shared memory each); large ones one per SM, and
-  // then a split only pays while all its CTAs fit in one wave.
-  if (n_pad > 96 && g.tiles * splits > 148) splits = 148 / g.tiles > 0 ? 148 / g.tiles : 1;
-  const bool two_per_sm = n_pad <= 96 && g.tiles * splits > 148;
+  // Blocks of up to 128 padded rows run two CTAs per SM (half the shared memory each: 4 ring stages
+  // up to 96 rows, 3 beyond); larger ones one per SM, and then a split only pays while all its CTAs
+  // fit in one wave.
+  if (n_pad > 128 && g.tiles * splits > 148) splits = 148 / g.tiles > 0 ? 148 / g.tiles : 1;
+  const bool two_per_sm = n_pad <= 128 && g.tiles * splits > 148;
   const size_t budget = (two_per_sm ? 110 : 220) * 1024;
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;

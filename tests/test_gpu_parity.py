@@ -20,7 +20,7 @@ def test_generators_are_bit_identical_on_cpu_and_gpu():
 # ------------------------------------------------------------------ single operators
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (19, 1376, 256), (19, 256, 688), (69, 1000, 4096),
-                                   (133, 384, 1024), (256, 130, 520)])
+                                   (133, 384, 1024), (256, 130, 520), (105, 4096, 4096), (128, 4096, 2048)])
 def test_projection_matches_fp64_matmul(M, N, K):
     from paper_2401_12522_b200 import bita_gemm_bf16
     X = synth.pseudo_normal(3, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda:0")
