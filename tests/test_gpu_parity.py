@@ -97,6 +97,7 @@ def test_tiny_config_lockstep_32_steps():
 TEMPLATES = {
     "comb-n3k5-pernode": (lambda: synth.comb_template(3, 5), 3),
     "comb-n4k3-pernode": (lambda: synth.comb_template(4, 3), 4),
+    "comb-n4k5-pernode": (lambda: synth.comb_template(4, 5), 4),     # 105 rows: past 96, one row tile
     "chain": (lambda: synth.chain_template(3), 3),
     "empty": (lambda: synth.empty_template(), 3),
     "product-pernode": (lambda: synth.product_rule_template((3, 3, 3), (3, 3, 3), per_node_groups=True), 3),
@@ -207,13 +208,15 @@ def test_errors_are_reported_not_raised_by_the_device():
 
 # ------------------------------------------------------------------ full-width shapes (the launch shapes bench.py times)
 
-@pytest.mark.parametrize("name,layers,prompt_len", [("7b", 2, 150), ("13b", 1, 140), ("70b", 1, 70)])
-def test_full_width_shapes_lockstep(name, layers, prompt_len):
+@pytest.mark.parametrize("name,layers,prompt_len,comb", [("7b", 2, 150, False), ("13b", 1, 140, False),
+                                                         ("70b", 1, 70, False), ("7b", 1, 120, True)])
+def test_full_width_shapes_lockstep(name, layers, prompt_len, comb):
     """Model width, head layout, FFN width, vocabulary, tree and block size of the measured configs;
     only the depth is cut so that the fp64 oracle finishes in seconds.  Every kernel runs in the
     grid/cluster/tile configuration of the full-depth step (none depends on the layer count)."""
     shape = synth.CONFIGS[name].with_layers(layers)
-    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    # comb: the paper's default tree (k = 5 candidates per depth, a mask group per node): 105 rows
+    tmpl = synth.comb_template(shape.n_mask, 5) if comb else synth.product_rule_template(shape.tree_K, shape.tree_B)
     seed = 0x5EED0010
     prompt = prompt_tokens(seed, prompt_len, shape.V)
     ref_model = oracle_model(shape, seed, lazy=True)
