@@ -34,6 +34,18 @@ METRIC = "accepted_tokens_per_s"
 UNIT = "tokens/s"
 
 
+# DRAM bytes (read + write) per projection launch at the 7B width with the 69-row block, from the ncu
+# capture summarised in profiles/k_gemm_tc_k_attn_umma_7b_ncu_full.md (q/k/v, O, gate/up, down per
+# layer; LM head).  Other shapes have no capture: their `traffic` is null.
+NCU_TRAFFIC_7B = {"per_layer": 105.79e6 + 35.51e6 + 185.17e6 + 97.30e6, "head": 266.42e6}
+
+
+def _traffic_per_mean_launch(shape, tmpl):
+    if not shape.name.startswith("7b") or (1 + tmpl.N + tmpl.G * shape.n_mask) != 69:
+        return None
+    return (shape.L * NCU_TRAFFIC_7B["per_layer"] + NCU_TRAFFIC_7B["head"]) / (4 * shape.L + 1)
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -348,7 +360,8 @@ def run_ours(args, shape, tmpl):
             "step_hbm_frac": (step_bytes / (step_ms * 1e-3) / 1e9) / peak,
             "roofline": {"bound": "hbm", "kernel": "projection (weight-streaming GEMM), mean over the step's launches",
                          "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None,
+                         "frac": achieved / peak, "algorithmic_bytes_per_launch": gemm_bytes,
+                         "traffic": _traffic_per_mean_launch(shape, tmpl),
                          "attention_ms_per_step": fam_ms[1] / n_prof, "projection_ms_per_step": fam_ms[0] / n_prof},
         }
         if world == 1 and not args.no_cpu_baseline:
