@@ -459,7 +459,7 @@ def run_next_rows(args, shape):
         C_max = shape.prompt_len + (steps + 8) * (depth + 1) + rows + 64
         ctx = Bita(shape, weights, tmpl, C_max=C_max, device=dev)
         ctx.reset()
-        # ---- first pass: chunks of 128 rows through the same kernels, then the first tree
+        # ---- first pass: equal blocks of up to 248 rows through the same kernels, then the first tree
         times = []
         for it in range(3):
             ctx.reset()

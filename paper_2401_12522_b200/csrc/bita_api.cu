@@ -59,7 +59,7 @@ int launch(cudaStream_t s, bool pdl, dim3 grid, dim3 block, size_t smem, unsigne
   return BITA_OK;
 }
 
-constexpr int PREFILL_CHUNK = 128;
+constexpr int PREFILL_CHUNK = BITA_MAX_ROWS - BITA_MAX_MASK;   // query rows per block of the first pass
 constexpr size_t ALIGN = 256;
 
 inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
@@ -779,8 +779,10 @@ int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count,
     if (tokens[i] < 0 || tokens[i] >= c->m.V) return BITA_ERR_INVALID_ARG;
   if ((long)c->len_upper + count + c->n_mask > kv->C_max) return BITA_ERR_KV_FULL;
   c->launches = 0;
-  for (int done = 0; done < count;) {
-    const int cnt = count - done < PREFILL_CHUNK ? count - done : PREFILL_CHUNK;
+  // Equal blocks, as few as the row limit allows: every block streams all the weights once.
+  int blocks_left = (count + PREFILL_CHUNK - 1) / PREFILL_CHUNK;
+  for (int done = 0; done < count; --blocks_left) {
+    const int cnt = (count - done + blocks_left - 1) / blocks_left;
     const bool last = done + cnt == count;
     build_prefill_plan(cnt, c->n_mask, last, c->step_plan.k_max, &c->prefill_plan);
     int rc = upload_plan(&c->prefill_plan, c->b.plan_prefill, c->stream);
