@@ -127,10 +127,15 @@ class Lockstep:
         rec_o = orc.prefill(self.model, self.blk, self.st, prompt)
         T = len(prompt)
         n = self.shape.n_mask
-        chunk = 128
-        last_start = ((T - 1) // chunk) * chunk
+        # the library runs the first pass in equal blocks of at most MAX_ROWS - 8 query rows; the debug
+        # buffers hold the last block only
+        from paper_2401_12522_b200 import MAX_ROWS
+        cap = MAX_ROWS - 8
+        blocks_left, last_start = -(-T // cap), 0
+        while blocks_left > 1:
+            last_start += -(-(T - last_start) // blocks_left)
+            blocks_left -= 1
         rows = T - last_start + n
-        # the debug buffers hold the last chunk only
         sub = dict(hidden=[h[last_start:] for h in rec_o["hidden"]], logits=rec_o["logits"][last_start:])
         gl, tol = self._compare_float(sub, rows)
         ol = sub["logits"]

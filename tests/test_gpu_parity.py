@@ -20,7 +20,8 @@ def test_generators_are_bit_identical_on_cpu_and_gpu():
 # ------------------------------------------------------------------ single operators
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (19, 1376, 256), (19, 256, 688), (69, 1000, 4096),
-                                   (133, 384, 1024), (256, 130, 520), (105, 4096, 4096), (128, 4096, 2048)])
+                                   (133, 384, 1024), (256, 130, 520), (105, 4096, 4096), (128, 4096, 2048),
+                                   (154, 4096, 4096), (200, 1000, 11008), (256, 12288, 4096)])
 def test_projection_matches_fp64_matmul(M, N, K):
     from paper_2401_12522_b200 import bita_gemm_bf16
     X = synth.pseudo_normal(3, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda:0")
@@ -81,6 +82,18 @@ def test_tree_attention_matches_oracle(B, N, H, H_kv, D, P, C):
 
 
 # ------------------------------------------------------------------ the whole pass, lockstep
+
+@pytest.mark.parametrize("plen", [140, 300])
+def test_first_pass_in_several_blocks(plen):
+    """Prompts longer than one block of the first pass (248 query rows): 140 tokens make one block of
+    143 rows (past 128: two attention row tiles), 300 make two blocks of 150."""
+    shape = synth.CONFIGS["tiny"]
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    seed = 0x5EED0777
+    ls = run_lockstep(shape, seed, tmpl, 3, prompt=prompt_tokens(seed, plen, shape.V))
+    assert ls.max_logit <= 3e-2
+    ls.close()
+
 
 def test_tiny_config_lockstep_32_steps():
     shape = synth.CONFIGS["tiny"]
