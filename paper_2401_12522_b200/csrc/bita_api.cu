@@ -272,8 +272,6 @@ int make_map3(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64
 struct GemmDesc {
   CUtensorMap a0, a1;
   int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
-  const void* w[2] = {nullptr, nullptr};   // the matrices themselves (for L2 prefetch by the previous projection)
-  size_t bytes = 0;                        // bytes of each
 };
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
@@ -294,9 +292,6 @@ int gemm_splits(int tiles, int K, int max_splits) {
 int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
   g->K = K;
   g->dual = W1 ? 1 : 0;
-  g->w[0] = W0;
-  g->w[1] = W1;
-  g->bytes = (size_t)N * K * 2;
   int rc;
   if (W1) {           // N = rows of each of the two matrices
     g->tiles = (N + 63) / 64;

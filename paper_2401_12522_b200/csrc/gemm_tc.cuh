@@ -9,20 +9,22 @@
 // blocks (split-K); it streams its weight tiles through a ring of TMA-filled, 128-byte-swizzled
 // shared-memory stages, one elected thread issues tcgen05.mma into a TMEM accumulator, and four
 // epilogue warps read the accumulator back with tcgen05.ld.  With split-K every split stores its
-// partial tile in an L2-resident exchange buffer and bumps a per-tile counter; the split that
-// completes the counter sums the partial tiles, always in split order - every output is a
-// fixed-order sum (deterministic, and independent of how many other rows the block holds), no CTA
-// waits for another, and the splits that are not last leave at once, which frees their SM for the
-// next kernel's prologue.  The reducing CTA then applies the fused operation: plain fp32 store; SwiGLU ("dual" mode
-// builds the 128-row weight tile from 64 gate rows and the 64 matching up rows, so both halves of
-// a product sit in the same tile); or rotary embedding with the q rows going to a bf16 buffer and
-// the k/v rows straight into the KV cache.
+// partial tile in an L2-resident exchange buffer and counts itself in on a per-tile counter; once
+// all splits of the tile are in, each of them sums an equal share of the tile's rows over the
+// partial tiles, always in split order - every output is a fixed-order sum (deterministic, and
+// independent of how many other rows the block holds) - and applies the fused operation to those
+// rows.  The splits of a launch run in one wave (the host sizes the grid so) and none waits before
+// its own partial tile is published, so the wait ends; it is bounded all the same.  Fused
+// operations: plain fp32 store; SwiGLU ("dual" mode builds the 128-row weight tile from 64 gate
+// rows and the 64 matching up rows, so both halves of a product sit in the same tile); rotary
+// embedding with the q rows going to a bf16 buffer and the k/v rows straight into the KV cache;
+// residual add with the next RMSNorm's input and row statistics.
 //
 // Programmatic dependent launch: the weight tiles of the first ring fill are requested before
 // the kernel waits for its predecessor, so HBM stays busy across the kernel boundary.
 //
-// Every wait on an mbarrier is bounded: when the bound is hit the kernel raises the status word,
-// lets its copies land, frees its TMEM and returns.
+// Every wait (mbarrier, split counter) is bounded: when the bound is hit the kernel raises the
+// status word, lets its copies land, frees its TMEM and returns.
 #pragma once
 
 #include <cuda.h>
