@@ -276,12 +276,27 @@ struct GemmDesc {
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
-constexpr int GEMM_MAX_CTAS = 296;
+constexpr int GEMM_MAX_CTAS = 296;       // size of the exchange buffer: two CTAs on each of up to 148 SMs
 constexpr int GEMM_MAX_SPLITS = 8;
+
+// SMs of the current device (the splits of a launch wait for one another, so a launch with splits
+// never has more CTAs than the GPU holds at once); capped at what the exchange buffer is sized for.
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v > GEMM_MAX_CTAS / 2 ? GEMM_MAX_CTAS / 2 : v;
+    else
+      n = 1;
+  }
+  return n;
+}
 
 int gemm_splits(int tiles, int K, int max_splits) {
   const int kb = (K + TC_BLOCK_K - 1) / TC_BLOCK_K;
-  int s = GEMM_MAX_CTAS / tiles;
+  int s = 2 * sm_count() / tiles;
   if (s > kb / 4) s = kb / 4;
   if (s > max_splits) s = max_splits;
   if (s > GEMM_MAX_SPLITS) s = GEMM_MAX_SPLITS;
@@ -325,8 +340,9 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   // Blocks of up to 128 padded rows run two CTAs per SM (half the shared memory each: 4 ring stages
   // up to 96 rows, 3 beyond); larger ones one per SM, and then a split only pays while all its CTAs
   // fit in one wave.
-  if (n_pad > 128 && g.tiles * splits > 148) splits = 148 / g.tiles > 0 ? 148 / g.tiles : 1;
-  const bool two_per_sm = n_pad <= 128 && g.tiles * splits > 148;
+  const int sms = sm_count();
+  if (n_pad > 128 && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
+  const bool two_per_sm = n_pad <= 128 && g.tiles * splits > sms;
   const size_t budget = (two_per_sm ? 110 : 220) * 1024;
   int stages = (int)((budget - 1024) / stage);
   if (stages > 10) stages = 10;
