@@ -447,7 +447,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
       for (int j = 0; j < 96; ++j)
         if (j < groups * 32 && c + j < p.M) dst[(c + j) * TC_BLOCK_N + fr] = v[j];
     }
-    if (p.splits > 1) __threadfence();
   }
   tc_fence_before();
   __syncthreads();
@@ -461,6 +460,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     if (threadIdx.x == 0) {
       // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
       // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+      __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
       atomicAdd(arrived, 1);
       unsigned long long w0 = 0;
       bool ok = true;
