@@ -2,7 +2,7 @@
 //
 // One CTA = one query head x one key slice x up to 128 query rows (arguments, slicing and the
 // partial-result format: attention_common.cuh).  The slice's keys are walked in chunks of 128; the
-// cache chunks come first, the prompt-prefix chunk last:
+// cache chunks come first, the prompt-prefix chunk last; slice s takes chunks s, s + S, ...:
 //   S = Q K^T      one UMMA chain, M = 128 (query rows), N = 128 (keys), K = D; Q and the K chunk
 //                  sit in shared memory as K-major 128-byte-swizzled tiles; S lands in TMEM with
 //                  lane = query row, column = key (two S buffers alternate);
@@ -182,20 +182,20 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   const int cache_chunks = (n_cache + AU_KEYS - 1) / AU_KEYS;
   const bool has_prompt = a.P > 0 && a.prompt_k && a.prompt_v && a.sees_prompt;
   const int n_chunks = cache_chunks + (has_prompt ? 1 : 0);
-  // Slice boundaries rounded up: the surplus chunks go to the first slices, so the last ones, which
-  // hold the block's own keys (not available before the dependency wait), have the least to do.
-  const int c_begin = (int)(((long)n_chunks * s + a.S - 1) / a.S);
-  const int c_end = (int)(((long)n_chunks * (s + 1) + a.S - 1) / a.S);
-  const int n = c_end - c_begin;
+  // Chunks are dealt round-robin: slice s takes chunks s, s + S, s + 2S, ...  The chunks that hold
+  // the block's own keys (the last cache chunks: not available before the dependency wait) thus go
+  // to different slices, each of which has earlier chunks to work on first.
+  const int n = s < n_chunks ? (n_chunks - s + a.S - 1) / a.S : 0;
+  auto chunk_of = [&](int i) { return s + i * a.S; };
   // The cache chunk that holds the last key may end in slots that were never written: their V rows
   // are cleared before the P V product (`fix` = index of that chunk within this slice, or -1).
-  const int fix = (n_cache % AU_KEYS != 0 && cache_chunks - 1 >= c_begin && cache_chunks - 1 < c_end)
-                      ? cache_chunks - 1 - c_begin : -1;
+  const int fix = (n_cache % AU_KEYS != 0 && cache_chunks - 1 >= s && (cache_chunks - 1 - s) % a.S == 0)
+                      ? (cache_chunks - 1 - s) / a.S : -1;
 
   if (warp == 5) {
     // ---------------- loader (one lane issues; the warp clears the rows of the `fix` chunk)
     auto issue_tile = [&](int i, bool v_tile) {                  // lane 0 only
-      const int ci = c_begin + i;
+      const int ci = chunk_of(i);
       const uint32_t dst = kv_s + (uint32_t)(i & 1) * 2 * TILE + (v_tile ? TILE : 0);
       const bool is_prompt = ci >= cache_chunks;
       const uint32_t bar = smem_u32(v_tile ? &bar_v_full[i & 1] : &bar_k_full[i & 1]);
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         tma_load_3d(dst + hf * AU_ATOM, map, hf * 64, is_prompt ? 0 : ci * AU_KEYS, is_prompt ? kvh : b * a.H_kv + kvh, bar);
     };
     // chunks without block rows depend on nothing the previous kernel writes
-    auto early = [&](int i) { const int ci = c_begin + i; return ci >= cache_chunks || (ci + 1) * AU_KEYS <= C; };
+    auto early = [&](int i) { const int ci = chunk_of(i); return ci >= cache_chunks || (ci + 1) * AU_KEYS <= C; };
     int k_issued = 0, v_issued = 0;
     while (k_issued < n && k_issued < 2 && early(k_issued)) {
       if (lane == 0) { issue_tile(k_issued, false); issue_tile(k_issued, true); }
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         ok = mbar_wait(smem_u32(&bar_v_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        const int live_rows = n_cache - (c_begin + j) * AU_KEYS;
+        const int live_rows = n_cache - chunk_of(j) * AU_KEYS;
         const uint32_t vs = kv_s + (uint32_t)(j & 1) * 2 * TILE + TILE;
         for (int t = lane; t < (AU_KEYS - live_rows) * CH; t += 32) {
           const int r = live_rows + t / CH, c = t % CH;
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int i = 0; i < n; ++i) {
-      const int ci = c_begin + i;
+      const int ci = chunk_of(i);
       const bool is_prompt = ci >= cache_chunks;
       const int key0 = is_prompt ? 0 : ci * AU_KEYS;
       const bool all_vis = !is_prompt && key0 + AU_KEYS <= C && row_live;
