@@ -358,7 +358,7 @@ def run_ours(args, shape, tmpl):
             "gpu_launches": launches,
             "clocks": clocks,
             "step_hbm_frac": (step_bytes / (step_ms * 1e-3) / 1e9) / peak,
-            "roofline": {"bound": "hbm", "kernel": "projection (weight-streaming GEMM), mean over the step's launches",
+            "roofline": {"bound": "hbm", "kernel": "projection (weight-streaming GEMM), mean over the step's launches; events at the boundaries of runs of consecutive projections",
                          "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                          "frac": achieved / peak, "algorithmic_bytes_per_launch": gemm_bytes,
                          "traffic": _traffic_per_mean_launch(shape, tmpl),

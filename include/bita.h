@@ -159,9 +159,10 @@ int bita_rewind(bita_ctx* ctx, bita_kv* kv, int32_t new_len, int32_t last_token)
  * `bytes` must hold L * BITA_MAX_ROWS * d + BITA_MAX_ROWS * V floats. */
 int bita_set_debug_buffer(bita_ctx* ctx, void* dev_buf, size_t bytes);
 
-/* Per-kernel-family device timing of later passes, for roofline reports.  When on, every
- * projection launch and every attention launch of a pass is bracketed by CUDA events on the
- * context's stream (a pass then runs its launches one by one instead of as one replayed graph).
+/* Per-kernel-family device timing of later passes, for roofline reports.  When on, a pass records
+ * a CUDA event on the context's stream wherever the kernel family changes, so that every run of
+ * consecutive launches of one family (e.g. O, gate/up, down and the next layer's q/k/v projection)
+ * is timed as a whole, overlapping as it does in an untimed pass.
  * bita_get_kernel_timing waits for the stream and returns, for the most recent pass, the summed
  * milliseconds and launch counts per family into HOST arrays of BITA_TIMING_FAMILIES entries:
  * [0] projections (QKV, O, gate/up, down, LM head), [1] tree attention. */

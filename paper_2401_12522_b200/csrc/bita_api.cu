@@ -447,31 +447,31 @@ struct bita_ctx {
   // optional per-family event timing
   bool timing;
   std::vector<cudaEvent_t> ev;          // pairs (start, stop)
-  std::vector<int> ev_family;           // family of each pair used by the last pass
+  std::vector<int> ev_family;           // timing: family of the run of launches that follows event i (-1 = end)
+  std::vector<int> ev_count;            // launches in that run
 };
 
 namespace {
 
-// Event bracket around one launch when timing is on.
-struct Timed {
-  bita_ctx* c;
-  int slot;
-  Timed(bita_ctx* ctx, int family) : c(ctx), slot(-1) {
-    if (!c->timing) return;
-    slot = (int)c->ev_family.size();
-    if ((size_t)(2 * slot + 1) >= c->ev.size()) {
-      cudaEvent_t a = nullptr, b = nullptr;
-      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { slot = -1; return; }
-      c->ev.push_back(a);
-      c->ev.push_back(b);
+// Timing marks: one event wherever the kernel family changes, so that a run of consecutive
+// launches of one family (e.g. O, gate/up, down and the next q/k/v projection) is timed as it
+// runs in an untimed pass, with each kernel's first weight tiles requested during its predecessor's
+// tail.  Families: 0 projections, 1 attention, 2 everything else, -1 closes the pass.
+void mark(bita_ctx* c, int family) {
+  if (!c->timing) return;
+  if (c->ev_family.empty() || c->ev_family.back() != family) {
+    const size_t i = c->ev_family.size();
+    if (i >= c->ev.size()) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->ev.push_back(e);
     }
+    cudaEventRecord(c->ev[i], c->stream);
     c->ev_family.push_back(family);
-    cudaEventRecord(c->ev[2 * slot], c->stream);
+    c->ev_count.push_back(0);
   }
-  ~Timed() {
-    if (slot >= 0) cudaEventRecord(c->ev[2 * slot + 1], c->stream);
-  }
-};
+  if (family >= 0) c->ev_count.back() += 1;
+}
 
 // Projection of the first M rows of an activation buffer (BITA_MAX_ROWS rows allocated).
 int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
@@ -487,7 +487,7 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   p.status = &c->b.state->status;
   p.part = c->b.gemm_part;
   p.tile_counters = c->b.gemm_cnt;
-  Timed t(c, 0);
+  mark(c, 0);
   int rc = launch_gemm_tc(g, it->second, n_pad, M, p, c->pdl, c->stream);
   c->launches++;
   return rc;
@@ -570,6 +570,8 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   cudaStream_t s = c->stream;
   Buffers& b = c->b;
   c->ev_family.clear();
+  c->ev_count.clear();
+  mark(c, 2);
   const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
   const bool pdl = c->pdl;
   int rc;
@@ -623,7 +625,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
     a.status = &b.state->status;
     {
-      Timed t(c, 1);
+      mark(c, 1);
       int n = 0;
       if ((rc = launch_attention(a, pdl, s, &n, &c->attn_map_cache))) return rc;
       c->launches += n;
@@ -645,6 +647,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
         CU_TRY(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         sel_attr = true;
       }
+      mark(c, 2);
       if ((rc = launch(s, pdl, dim3(M), dim3(1024), use_smem ? row_bytes : 0, 1, k_select, P, (const float*)b.logits,
                        m.V, use_smem, b.sel_id, b.sel_val)))
         return rc;
@@ -654,6 +657,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
       CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,
                              cudaMemcpyDeviceToDevice, s));
   }
+  mark(c, -1);
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }
@@ -881,11 +885,13 @@ int bita_get_kernel_timing(bita_ctx* c, float* ms, int32_t* launches) {
   if (!c || !ms || !launches) return BITA_ERR_INVALID_ARG;
   CU_TRY(cudaStreamSynchronize(c->stream));
   for (int f = 0; f < BITA_TIMING_FAMILIES; ++f) { ms[f] = 0.f; launches[f] = 0; }
-  for (size_t i = 0; i < c->ev_family.size(); ++i) {
+  for (size_t i = 0; i + 1 < c->ev_family.size(); ++i) {
+    const int f = c->ev_family[i];
+    if (f < 0 || f >= BITA_TIMING_FAMILIES) continue;
     float t = 0.f;
-    CU_TRY(cudaEventElapsedTime(&t, c->ev[2 * i], c->ev[2 * i + 1]));
-    ms[c->ev_family[i]] += t;
-    launches[c->ev_family[i]] += 1;
+    CU_TRY(cudaEventElapsedTime(&t, c->ev[i], c->ev[i + 1]));
+    ms[f] += t;
+    launches[f] += c->ev_count[i];
   }
   return BITA_OK;
 }
