@@ -67,127 +67,82 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
 
 // ---------------------------------------------------------------------------------------------
 // Argmax / sorted top-k of each logits row, order = (value descending, token id ascending).
-// One block per row.  Rows that need only the argmax take one pass over the row.  Mask rows (top
-// k_max): the row is copied to shared memory (when it fits), every warp then finds the sorted
-// top-K of its own contiguous segment in K warp-local rounds (round t = best entry strictly after
-// the warp's previous pick), and one warp merges the warps' candidates the same way; the global
-// top-K is among them.
+// One block per row; pass t picks the best entry strictly after the previous pick.
 // sel_id: int32 [M][BITA_MAX_TOPK], sel_val: fp32 [M][BITA_MAX_TOPK].
 __device__ __forceinline__ bool before(float v1, int i1, float v2, int i2) {
   return v1 > v2 || (v1 == v2 && i1 < i2);
-}
-__device__ __forceinline__ void warp_best(float& bv, int& bi) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-  }
 }
 
 __global__ void __launch_bounds__(1024) k_select(DevPlan plan, const float* __restrict__ logits, int V, int use_smem,
                                                  int32_t* __restrict__ sel_id, float* __restrict__ sel_val) {
   pdl_launch();
   pdl_wait();
-  extern __shared__ float srow[];            // the row, kept on chip for the warp-local rounds (when it fits)
-  __shared__ float cv[32][BITA_MAX_TOPK];    // candidates of each warp, sorted
-  __shared__ int ci[32][BITA_MAX_TOPK];
+  extern __shared__ float srow[];            // the row, kept on chip for the later passes (when it fits)
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  __shared__ float pv;
+  __shared__ int pi;
   const int r = blockIdx.x;
   const int kind = plan.row_kind[r];
   const int K = (kind == ROW_MASK) ? plan.k_max : 1;
   const float* row = logits + (size_t)r * V;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  const bool vec = (V & 3) == 0;
-  constexpr int NONE = 0x7fffffff;
-
-  if (K == 1) {
-    // ---- argmax: one pass, 16-byte loads
+  float prev_v = 0.f;
+  int prev_i = -1;
+  for (int t = 0; t < K; ++t) {
     float bv = -INFINITY;
-    int bi = NONE;
-    if (vec) {
+    int bi = 0x7fffffff;
+    if (t == 0 && (V & 3) == 0) {
+      // first pass: 16-byte loads from global memory, copy to shared memory on the way
       const float4* row4 = reinterpret_cast<const float4*>(row);
       for (int c4 = threadIdx.x; c4 < (V >> 2); c4 += blockDim.x) {
         const float4 q = row4[c4];
+        if (use_smem && K > 1) reinterpret_cast<float4*>(srow)[c4] = q;
         const float vals[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (vals[e] == vals[e] && before(vals[e], 4 * c4 + e, bv, bi)) { bv = vals[e]; bi = 4 * c4 + e; }
+        for (int e = 0; e < 4; ++e) {
+          const float v = vals[e];
+          const int c = 4 * c4 + e;
+          if (v == v && before(v, c, bv, bi)) { bv = v; bi = c; }
+        }
       }
     } else {
+      const float* src = (t > 0 && use_smem && (V & 3) == 0) ? srow : row;
       for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        const float v = row[c];
-        if (v == v && before(v, c, bv, bi)) { bv = v; bi = c; }
-      }
-    }
-    warp_best(bv, bi);
-    if (lane == 0) { cv[warp][0] = bv; ci[warp][0] = bi; }
-    __syncthreads();
-    if (warp == 0) {
-      bv = lane < nw ? cv[lane][0] : -INFINITY;
-      bi = lane < nw ? ci[lane][0] : NONE;
-      warp_best(bv, bi);
-      if (lane == 0) {
-        sel_id[(size_t)r * BITA_MAX_TOPK] = bi == NONE ? -1 : bi;
-        sel_val[(size_t)r * BITA_MAX_TOPK] = bv;
-      }
-    }
-    return;
-  }
-
-  // ---- sorted top-K
-  const bool on_chip = use_smem && vec;
-  if (on_chip) {
-    const float4* row4 = reinterpret_cast<const float4*>(row);
-    for (int c4 = threadIdx.x; c4 < (V >> 2); c4 += blockDim.x) reinterpret_cast<float4*>(srow)[c4] = row4[c4];
-    __syncthreads();
-  }
-  const float* src = on_chip ? srow : row;
-  const int seg = (V + nw - 1) / nw;
-  const int lo = warp * seg, hi = min(V, lo + seg);
-  float prev_v = 0.f;
-  int prev_i = -1;                            // -1: nothing picked yet
-  for (int t = 0; t < K; ++t) {
-    float bv = -INFINITY;
-    int bi = NONE;
-    if (prev_i != NONE) {                     // NONE: the segment is exhausted
-      for (int c = lo + lane; c < hi; c += 32) {
         const float v = src[c];
         if (!(v == v)) continue;
-        if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;   // not strictly after the previous pick
+        if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;  // not strictly after the previous pick
         if (before(v, c, bv, bi)) { bv = v; bi = c; }
       }
-      warp_best(bv, bi);
     }
-    if (lane == 0) { cv[warp][t] = bv; ci[warp][t] = bi; }
-    prev_v = bv;
-    prev_i = bi;
-  }
-  __syncthreads();
-  if (warp == 0) {
-    // merge: K rounds over the nw * K candidates (lane owns candidates lane, lane + 32, ...)
-    const int n_c = nw * K;
-    float gv = 0.f;
-    int gi = -1;
-    for (int t = 0; t < K; ++t) {
-      float bv = -INFINITY;
-      int bi = NONE;
-      if (gi != NONE) {
-        for (int e = lane; e < n_c; e += 32) {
-          const float v = cv[e / K][e % K];
-          const int c = ci[e / K][e % K];
-          if (c == NONE) continue;
-          if (gi >= 0 && !before(gv, gi, v, c)) continue;
-          if (before(v, c, bv, bi)) { bv = v; bi = c; }
-        }
-        warp_best(bv, bi);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int nw = blockDim.x >> 5;
+      bv = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+      bi = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
       }
-      if (lane == 0) {
-        sel_id[(size_t)r * BITA_MAX_TOPK + t] = bi == NONE ? -1 : bi;
+      if (threadIdx.x == 0) {
+        pv = bv;
+        pi = (bi == 0x7fffffff) ? -1 : bi;
+        sel_id[(size_t)r * BITA_MAX_TOPK + t] = pi;
         sel_val[(size_t)r * BITA_MAX_TOPK + t] = bv;
       }
-      gv = bv;
-      gi = bi;
     }
+    __syncthreads();
+    prev_v = pv;
+    prev_i = pi;
+    if (prev_i < 0) break;
   }
 }
 
