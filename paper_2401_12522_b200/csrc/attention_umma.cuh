@@ -1,6 +1,7 @@
 // Tree-based attention (Sec. 3.2, Fig. 6) on the tcgen05 tensor cores.
 //
-// One CTA = one query head x one key slice x up to 128 query rows (arguments, slicing and the
+// One CTA = one query head x one key slice x RT row tiles of 128 query rows (RT = 2 for blocks of
+// more than 128 rows, so that both tiles share every K/V chunk that is read; arguments, slicing and the
 // partial-result format: attention_common.cuh).  The slice's keys are walked in chunks of 128; the
 // cache chunks come first, the prompt-prefix chunk last; slice s takes chunks s, s + S, ...:
 //   S = Q K^T      one UMMA chain, M = 128 (query rows), N = 128 (keys), K = D; Q and the K chunk
@@ -116,11 +117,12 @@ __device__ __forceinline__ uint32_t au_off(int r, int c) {
   return (uint32_t)((c >> 3) * AU_ATOM + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-template <int D>
+template <int D, int RT>
 __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_constant__ AttnMaps maps, AttnArgs a) {
   constexpr int CH = D / 8;                         // 16-byte chunks per row
   constexpr int TILE = (D / 64) * AU_ATOM;          // bytes of a staged [128][D] tile
-  constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;
+  constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;   // two S buffers, then RT output accumulators of D columns
+  static_assert(2 * AU_KEYS + RT * D <= 512, "tensor memory");
   constexpr uint32_t TMEM_COLS = 512;
   constexpr uint32_t PSTRIDE = (D + 4) * 4;         // bytes of a partial row in shared memory: m, l, pad, O[D]
   extern __shared__ uint8_t smem_raw[];
@@ -135,11 +137,12 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   const int h = blockIdx.x, s = blockIdx.y;
   const int b = blockIdx.z / a.row_tiles, rt = blockIdx.z - b * a.row_tiles;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = rt * AU_ROWS;
+  const int row0 = rt * RT * AU_ROWS;
   const int kvh = h / (a.H / a.H_kv);
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t q_s = base, kv_s = base + TILE, p_s = base + TILE + 4 * TILE;   // kv: 2 x (K tile, V tile)
+  // Q (RT tiles), 2 x (K tile, V tile), P
+  const uint32_t q_s = base, kv_s = base + RT * TILE, p_s = kv_s + 4 * TILE;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -187,6 +190,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   // to different slices, each of which has earlier chunks to work on first.
   const int n = s < n_chunks ? (n_chunks - s + a.S - 1) / a.S : 0;
   auto chunk_of = [&](int i) { return s + i * a.S; };
+  // The tensor core and the softmax warps work in steps j = chunk * RT + row tile; S buffer j & 1.
+  const int n_steps = n * RT;
   // The cache chunk that holds the last key may end in slots that were never written: their V rows
   // are cleared before the P V product (`fix` = index of that chunk within this slice, or -1).
   const int fix = (n_cache % AU_KEYS != 0 && cache_chunks - 1 >= s && (cache_chunks - 1 - s) % a.S == 0)
@@ -215,18 +220,21 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     v_issued = k_issued;
     pdl_wait();
     if (lane == 0 && n > 0) {
-      mbar_expect_tx(smem_u32(&bar_q), (uint32_t)TILE);
+      mbar_expect_tx(smem_u32(&bar_q), (uint32_t)(RT * TILE));
 #pragma unroll
-      for (int hf = 0; hf < D / 64; ++hf)
-        tma_load_3d(q_s + hf * AU_ATOM, &maps.q, hf * 64, h, b * a.M + row0, smem_u32(&bar_q));
+      for (int t = 0; t < RT; ++t) {
+#pragma unroll
+        for (int hf = 0; hf < D / 64; ++hf)
+          tma_load_3d(q_s + t * TILE + hf * AU_ATOM, &maps.q, hf * 64, h, b * a.M + row0 + t * AU_ROWS, smem_u32(&bar_q));
+      }
     }
     bool ok = true;
     if (k_issued == 0 && n > 0) {
       if (lane == 0) issue_tile(0, false);
       k_issued = 1;
     }
-    // The MMA thread runs S(0), S(1), PV(0), S(2), PV(1), ...: K(j+1) waits for S(j-1), then V(j)
-    // waits for PV(j-2), in that order.
+    // The MMA thread runs (per chunk, all row tiles) S(0), S(1), PV(0), S(2), PV(1), ...: K(j+1)
+    // waits for the S of chunk j-1, then V(j) for the PV of chunk j-2, in that order.
     for (int j = 0; j < n && ok; ++j) {
       if (j + 1 < n && j + 1 >= k_issued) {
         if (j + 1 >= 2) ok = mbar_wait(smem_u32(&bar_k_empty[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status);
@@ -266,34 +274,37 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       const uint32_t idesc_s = umma_idesc(AU_KEYS);                       // S: N = keys of a chunk
       const uint32_t idesc_o = umma_idesc(D) | (1u << 16);                // O: N = D, B operand MN-major
       bool ok = true;
-      auto issue_s = [&](int i) {
+      auto issue_s = [&](int j) {                                         // step j: chunk j / RT, row tile j % RT
+        const int i = j / RT, t = j - i * RT;
         const uint32_t ks = kv_s + (uint32_t)(i & 1) * 2 * TILE;
-        const uint32_t d_tmem = tmem + COL_S + (uint32_t)(i & 1) * AU_KEYS;
+        const uint32_t d_tmem = tmem + COL_S + (uint32_t)(j & 1) * AU_KEYS;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t da = umma_smem_desc(q_s + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
+          const uint64_t da = umma_smem_desc(q_s + t * TILE + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
           const uint64_t db = umma_smem_desc(ks + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
           umma_bf16(d_tmem, da, db, idesc_s, kk > 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bar_s_full[i & 1]));
-        umma_commit(smem_u32(&bar_k_empty[i & 1]));
+        umma_commit(smem_u32(&bar_s_full[j & 1]));
+        if (t == RT - 1) umma_commit(smem_u32(&bar_k_empty[i & 1]));      // the K tile has served every row tile
       };
       ok = mbar_wait(smem_u32(&bar_q), 0, status);
       if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, status);
       tc_fence_after();
       if (ok) issue_s(0);
-      for (int i = 0; i < n && ok; ++i) {
-        if (i + 1 < n) {                                                  // S of the next chunk while this one is in softmax
-          ok = mbar_wait(smem_u32(&bar_k_full[(i + 1) & 1]), (uint32_t)((i + 1) >> 1) & 1u, status);
-          if (ok && i + 1 >= 2)
-            ok = mbar_wait(smem_u32(&bar_s_free[(i + 1) & 1]), ((uint32_t)((i + 1) >> 1) & 1u) ^ 1u, status);
+      for (int j = 0; j < n_steps && ok; ++j) {
+        if (j + 1 < n_steps) {                                            // S of the next step while this one is in softmax
+          const int i1 = (j + 1) / RT;
+          if ((j + 1) % RT == 0) ok = mbar_wait(smem_u32(&bar_k_full[i1 & 1]), (uint32_t)(i1 >> 1) & 1u, status);
+          if (ok && j + 1 >= 2)
+            ok = mbar_wait(smem_u32(&bar_s_free[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status);
           if (!ok) break;
           tc_fence_after();
-          issue_s(i + 1);
+          issue_s(j + 1);
         }
-        ok = mbar_wait(smem_u32(&bar_p_full), (uint32_t)i & 1u, status);
-        if (ok) ok = mbar_wait(smem_u32(&bar_v_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
-        if (ok && i == fix) ok = mbar_wait(smem_u32(&bar_vfix), 0, status);
+        const int i = j / RT, t = j - i * RT;
+        ok = mbar_wait(smem_u32(&bar_p_full), (uint32_t)j & 1u, status);
+        if (ok && t == 0) ok = mbar_wait(smem_u32(&bar_v_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
+        if (ok && t == 0 && i == fix) ok = mbar_wait(smem_u32(&bar_vfix), 0, status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
@@ -301,44 +312,59 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         for (int kk = 0; kk < AU_KEYS / 16; ++kk) {
           const uint64_t da = umma_smem_desc(p_s + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
           const uint64_t db = umma_smem_desc_mn(vs + kk * 16 * 128, AU_ATOM);
-          umma_bf16(tmem + COL_O, da, db, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+          umma_bf16(tmem + COL_O + (uint32_t)(t * D), da, db, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bar_v_empty[i & 1]));
+        if (t == RT - 1) umma_commit(smem_u32(&bar_v_empty[i & 1]));
         umma_commit(smem_u32(&bar_pv_done));
       }
     }
   } else {
-    // ---------------- softmax: thread r owns query row r
+    // ---------------- softmax: thread r owns query row r of every row tile of the CTA
     const int r = threadIdx.x;
-    const int gr = row0 + r;
-    const bool row_live = gr < a.M;
     const float sc = a.scale_log2;
-    uint32_t visw[8];
+    int gr[RT];
+    bool row_live[RT], sees_p[RT];
+    uint32_t visw[RT][8];
+    float m_run[RT], l_run[RT];
 #pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      visw[w] = (row_live && w < a.W) ? a.vis[(size_t)b * a.vis_batch_stride + (size_t)gr * a.W + w] : 0u;
-      const int nb = a.M - 32 * w;                              // block rows this word can name
-      if (nb < 32) visw[w] &= nb <= 0 ? 0u : ((1u << nb) - 1u);
+    for (int t = 0; t < RT; ++t) {
+      gr[t] = row0 + t * AU_ROWS + r;
+      row_live[t] = gr[t] < a.M;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        visw[t][w] = (row_live[t] && w < a.W) ? a.vis[(size_t)b * a.vis_batch_stride + (size_t)gr[t] * a.W + w] : 0u;
+        const int nb = a.M - 32 * w;                            // block rows this word can name
+        if (nb < 32) visw[t][w] &= nb <= 0 ? 0u : ((1u << nb) - 1u);
+      }
+      sees_p[t] = has_prompt && row_live[t] && a.sees_prompt[(size_t)b * a.sp_batch_stride + gr[t]] != 0;
+      m_run[t] = -INFINITY;
+      l_run[t] = 0.f;
     }
-    const bool sees_p = has_prompt && row_live && a.sees_prompt[(size_t)b * a.sp_batch_stride + gr] != 0;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-    float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int i = 0; i < n; ++i) {
+    for (int j = 0; j < n_steps; ++j) {
+      const int i = j / RT;
       const int ci = chunk_of(i);
       const bool is_prompt = ci >= cache_chunks;
       const int key0 = is_prompt ? 0 : ci * AU_KEYS;
-      const bool all_vis = !is_prompt && key0 + AU_KEYS <= C && row_live;
+      // this step's row tile (compile-time selects keep the per-tile state in registers)
+      const bool second = RT > 1 && (j & 1);
+      const bool live = second ? row_live[RT - 1] : row_live[0];
+      const bool sp = second ? sees_p[RT - 1] : sees_p[0];
+      const float m_old = second ? m_run[RT - 1] : m_run[0];
+      const uint32_t o_addr = lane_addr + COL_O + (second ? (uint32_t)((RT - 1) * D) : 0u);
+      const uint32_t r_row = (uint32_t)r;
+      const bool all_vis = !is_prompt && key0 + AU_KEYS <= C && live;
       // Visibility of the chunk's 128 keys for this row as four 32-bit words: context keys are
       // seen by every live row, block keys according to the row's ancestor bitmask (shifted to the
       // key's place), prompt keys by mask rows only; keys past the last one by nobody.
       uint32_t vm[4] = {0u, 0u, 0u, 0u};
-      if (row_live && !all_vis) {
+      if (live && !all_vis) {
         if (is_prompt) {
 #pragma unroll
           for (int w = 0; w < 4; ++w) {
             const int nb = a.P - 32 * w;                        // prompt keys in this word
-            vm[w] = !sees_p || nb <= 0 ? 0u : (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u));
+            vm[w] = !sp || nb <= 0 ? 0u : (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u));
           }
         } else {
 #pragma unroll
@@ -352,9 +378,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
               const int q = j0 >= 0 ? j0 >> 5 : -1, sh = j0 & 31;
               uint32_t lo = q < 0 ? 0xffffffffu : 0u, hi = 0u;
 #pragma unroll
-              for (int t = 0; t < 8; ++t) {
-                if (t == q) lo = visw[t];
-                if (t == q + 1) hi = visw[t];
+              for (int u = 0; u < 8; ++u) {
+                const uint32_t vw = second ? visw[RT - 1][u] : visw[0][u];
+                if (u == q) lo = vw;
+                if (u == q + 1) hi = vw;
               }
               word = sh == 0 ? lo : __funnelshift_r(lo, hi, sh);
             }
@@ -362,31 +389,31 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           }
         }
       }
-      if (ok) ok = mbar_wait(smem_u32(&bar_s_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
+      if (ok) ok = mbar_wait(smem_u32(&bar_s_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
-      const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(i & 1) * AU_KEYS;
+      const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(j & 1) * AU_KEYS;
       // the whole row of scores into registers (one TMEM round trip); the buffer is free again
       float sv[AU_KEYS];
       tmem_ld128(s_addr, sv);
       tc_fence_before();
-      mbar_arrive_cta(smem_u32(&bar_s_free[i & 1]));
+      mbar_arrive_cta(smem_u32(&bar_s_free[j & 1]));
       float mx = -INFINITY;
       if (all_vis) {
 #pragma unroll
-        for (int j = 0; j < AU_KEYS; ++j) mx = fmaxf(mx, sv[j]);
+        for (int e = 0; e < AU_KEYS; ++e) mx = fmaxf(mx, sv[e]);
       } else {
 #pragma unroll
-        for (int j = 0; j < AU_KEYS; ++j) {
-          if (!((vm[j >> 5] >> (j & 31)) & 1u)) sv[j] = -INFINITY;   // exp2(-inf) = 0 below
-          mx = fmaxf(mx, sv[j]);
+        for (int e = 0; e < AU_KEYS; ++e) {
+          if (!((vm[e >> 5] >> (e & 31)) & 1u)) sv[e] = -INFINITY;   // exp2(-inf) = 0 below
+          mx = fmaxf(mx, sv[e]);
         }
       }
-      const float m_new = fmaxf(m_run, mx * sc);
+      const float m_new = fmaxf(m_old, mx * sc);
       const float sub = m_new == -INFINITY ? 0.f : m_new;
-      const float corr = exp2f(m_run - sub);                    // 0 while nothing was seen before
-      // P overwrites the tile the previous P V product reads, and the rescale touches its accumulator
-      if (i > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(i - 1) & 1u, status);
+      const float corr = exp2f(m_old - sub);                    // 0 while nothing was seen before
+      // P overwrites the tile the previous P V product reads, and the rescale touches an accumulator
+      if (j > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       // P = exp2(s * scale - max), row sum, bf16 tile
@@ -395,78 +422,81 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       for (int c0 = 0; c0 < AU_KEYS; c0 += 8) {
         uint32_t pk[4];
 #pragma unroll
-        for (int j = 0; j < 8; j += 2) {
-          const float p0 = ex2_approx(sv[c0 + j] * sc - sub), p1 = ex2_approx(sv[c0 + j + 1] * sc - sub);
+        for (int e = 0; e < 8; e += 2) {
+          const float p0 = ex2_approx(sv[c0 + e] * sc - sub), p1 = ex2_approx(sv[c0 + e + 1] * sc - sub);
           sum += p0 + p1;
-          pk[j >> 1] = pack_bf16x2(p0, p1);
+          pk[e >> 1] = pack_bf16x2(p0, p1);
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, c0 >> 3)), "r"(pk[0]), "r"(pk[1]),
-                     "r"(pk[2]), "r"(pk[3])
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off((int)r_row, c0 >> 3)), "r"(pk[0]),
+                     "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
                      : "memory");
       }
       if (i > 0 && __any_sync(0xffffffffu, corr != 1.0f)) {
         // the maximum of some row of this warp moved: bring the accumulator rows to their new
         // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch)
         float ov[D];
-        if constexpr (D == 128) tmem_ld128(lane_addr + COL_O, ov); else tmem_ld64(lane_addr + COL_O, ov);
+        if constexpr (D == 128) tmem_ld128(o_addr, ov); else tmem_ld64(o_addr, ov);
 #pragma unroll
-        for (int j = 0; j < D; ++j) ov[j] *= corr;
-        if constexpr (D == 128) tmem_st128(lane_addr + COL_O, ov); else tmem_st64(lane_addr + COL_O, ov);
+        for (int e = 0; e < D; ++e) ov[e] *= corr;
+        if constexpr (D == 128) tmem_st128(o_addr, ov); else tmem_st64(o_addr, ov);
       }
-      l_run = l_run * corr + sum;
-      m_run = m_new;
+      if (second) { l_run[RT - 1] = l_run[RT - 1] * corr + sum; m_run[RT - 1] = m_new; }
+      else { l_run[0] = l_run[0] * corr + sum; m_run[0] = m_new; }
       fence_async_smem();                                       // the P tile is read by the tensor core
       tc_fence_before();
       mbar_arrive_cta(smem_u32(&bar_p_full));
     }
-    if (n > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(n - 1) & 1u, status);
+    if (n_steps > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(n_steps - 1) & 1u, status);
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     pdl_wait();
-    // ---- result of this slice: row r of O
-    float ov[D];
-    if (n > 0 && ok) {
-      if constexpr (D == 128) tmem_ld128(lane_addr + COL_O, ov); else tmem_ld64(lane_addr + COL_O, ov);
-    } else {
+    // ---- result of this slice: row r of O, per row tile
 #pragma unroll
-      for (int j = 0; j < D; ++j) ov[j] = 0.f;
-    }
-    if (a.S == 1) {
-      const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-      if (row_live) {
-        bf16* dst = a.out + (((size_t)b * a.M + gr) * a.H + h) * D;
+    for (int t = 0; t < RT; ++t) {
+      float ov[D];
+      if (n_steps > 0 && ok) {
+        if constexpr (D == 128) tmem_ld128(lane_addr + COL_O + t * D, ov); else tmem_ld64(lane_addr + COL_O + t * D, ov);
+      } else {
 #pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 8) {
-          uint4 w;
-          w.x = pack_bf16x2(ov[c0] * inv, ov[c0 + 1] * inv);     w.y = pack_bf16x2(ov[c0 + 2] * inv, ov[c0 + 3] * inv);
-          w.z = pack_bf16x2(ov[c0 + 4] * inv, ov[c0 + 5] * inv); w.w = pack_bf16x2(ov[c0 + 6] * inv, ov[c0 + 7] * inv);
-          *reinterpret_cast<uint4*>(dst + c0) = w;
+        for (int e = 0; e < D; ++e) ov[e] = 0.f;
+      }
+      if (a.S == 1) {
+        const float inv = l_run[t] > 0.f ? 1.0f / l_run[t] : 0.f;
+        if (row_live[t]) {
+          bf16* dst = a.out + (((size_t)b * a.M + gr[t]) * a.H + h) * D;
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 8) {
+            uint4 w;
+            w.x = pack_bf16x2(ov[c0] * inv, ov[c0 + 1] * inv);     w.y = pack_bf16x2(ov[c0 + 2] * inv, ov[c0 + 3] * inv);
+            w.z = pack_bf16x2(ov[c0 + 4] * inv, ov[c0 + 5] * inv); w.w = pack_bf16x2(ov[c0 + 6] * inv, ov[c0 + 7] * inv);
+            *reinterpret_cast<uint4*>(dst + c0) = w;
+          }
+        }
+      } else if (a.cluster) {
+        // partial result of this row into this CTA's shared memory (the chunk buffers and the P tile
+        // are free: every copy into them has landed and every MMA that read them is complete)
+        if (row_live[t]) {
+          const uint32_t prow = kv_s + (uint32_t)(t * AU_ROWS + r) * PSTRIDE;
+          asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(prow), "f"(m_run[t]), "f"(l_run[t]) : "memory");
+#pragma unroll
+          for (int e = 0; e < D; e += 4)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(prow + 16 + e * 4), "f"(ov[e]), "f"(ov[e + 1]),
+                         "f"(ov[e + 2]), "f"(ov[e + 3])
+                         : "memory");
+        }
+      } else {
+        const size_t pbase = (((size_t)b * a.H + h) * a.S + s) * a.M;
+        if (row_live[t]) {
+          a.part_ml[(pbase + gr[t]) * 2] = m_run[t];
+          a.part_ml[(pbase + gr[t]) * 2 + 1] = l_run[t];
+          float* dst = a.part_acc + (pbase + gr[t]) * D;
+#pragma unroll
+          for (int e = 0; e < D; e += 4)
+            *reinterpret_cast<float4*>(dst + e) = make_float4(ov[e], ov[e + 1], ov[e + 2], ov[e + 3]);
         }
       }
-    } else if (a.cluster) {
-      // partial result of this row into this CTA's shared memory (the chunk buffers are free:
-      // every copy into them has landed and every MMA that read them is complete)
-      if (row_live) {
-        const uint32_t prow = kv_s + (uint32_t)r * PSTRIDE;
-        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(prow), "f"(m_run), "f"(l_run) : "memory");
-#pragma unroll
-        for (int j = 0; j < D; j += 4)
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(prow + 16 + j * 4), "f"(ov[j]), "f"(ov[j + 1]),
-                       "f"(ov[j + 2]), "f"(ov[j + 3])
-                       : "memory");
-      }
-    } else {
-      const size_t pbase = (((size_t)b * a.H + h) * a.S + s) * a.M;
-      if (row_live) {
-        a.part_ml[(pbase + gr) * 2] = m_run;
-        a.part_ml[(pbase + gr) * 2 + 1] = l_run;
-        float* dst = a.part_acc + (pbase + gr) * D;
-#pragma unroll
-        for (int j = 0; j < D; j += 4)
-          *reinterpret_cast<float4*>(dst + j) = make_float4(ov[j], ov[j + 1], ov[j + 2], ov[j + 3]);
-      }
-      __threadfence();
     }
+    if (a.S > 1 && !a.cluster) __threadfence();
   }
 
   // ---- merge inside the cluster: the S slices of this (sequence, head, row tile) are the CTAs of
@@ -483,7 +513,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
     mbar_wait_cluster(smem_u32(&bar_cl_in), 0, status);
     constexpr int VW = D / 32;
-    const int rows_here = min(AU_ROWS, a.M - row0);
+    const int rows_here = min(RT * AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
     constexpr int NW = AU_THREADS / 32, RR = 3;                 // rows per warp whose loads fly together
     for (int r0 = r_lo + warp; r0 < r_hi; r0 += NW * RR) {

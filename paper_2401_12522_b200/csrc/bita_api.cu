@@ -356,13 +356,14 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
 
 inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
 
-// Attention launch shape: row tiles of 128 query rows, and key slices.  The slices of a (sequence,
+// Attention launch shape: row tiles (one CTA takes one tile of 128 query rows, or two when the block
+// has more than 128 rows), and key slices.  The slices of a (sequence,
 // head, row tile) form a thread-block cluster; the slice count is the largest cluster size whose
 // clusters all fit the GPU at once (one CTA per SM; concurrent clusters seen on a B200: 74 of size
 // 2, 45 of 3, 33 of 4, 22 of 6, 15 of 8).  More clusters than that would still be correct (they
 // run in waves), just not faster.
 void attn_shape(int H, int B, int M, int* row_tiles, int* splits) {
-  const int rt = (M + AU_ROWS - 1) / AU_ROWS;
+  const int rt = (M + 2 * AU_ROWS - 1) / (2 * AU_ROWS);       // a CTA takes up to two tiles of 128 rows
   const int groups = H * B * rt;
   static const int size[5] = {8, 6, 4, 3, 2}, fit[5] = {15, 22, 33, 45, 74};
   int s = 1;
@@ -534,18 +535,24 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
     if (rc) return rc;
   }
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
+  const int RT = a.M > AU_ROWS ? 2 : 1;                          // row tiles per CTA
   const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
-  const size_t smem = 5 * tile + 2 * AU_ATOM + 1024;           // Q, 2 x (K, V), P
+  const size_t smem = (RT + 4) * tile + 2 * AU_ATOM + 1024;       // Q (RT tiles), 2 x (K, V), P
   static bool attr_set = false;
   if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     attr_set = true;
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
   auto run = [&](unsigned cluster_y) {
-    return a.D == 128 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<128>, maps, a)
-                      : launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<64>, maps, a);
+    if (a.D == 128)
+      return RT == 2 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<128, 2>, maps, a)
+                     : launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<128, 1>, maps, a);
+    return RT == 2 ? launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<64, 2>, maps, a)
+                   : launch(s, pdl, g1, dim3(AU_THREADS), smem, cluster_y, k_attn_umma<64, 1>, maps, a);
   };
   if (n_launched) *n_launched = 1;
   if (a.S == 1) return run(1);
