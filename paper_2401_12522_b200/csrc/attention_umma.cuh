@@ -7,15 +7,17 @@
 //   S = Q K^T      one UMMA chain, M = 128 (query rows), N = 128 (keys), K = D; Q and the K chunk
 //                  sit in shared memory as K-major 128-byte-swizzled tiles; S lands in TMEM with
 //                  lane = query row, column = key (two S buffers alternate);
-//   softmax        thread r of the four softmax warps owns query row r: it reads its row of S
-//                  from TMEM, applies the visibility rule (context / ancestor bitmask / prompt
-//                  prefix), keeps the running maximum and sum (online softmax, log2 domain),
-//                  writes P = exp2(..) as bf16 into a K-major shared-memory tile and, when the
-//                  maximum moved, rescales its row of the output accumulator in TMEM;
+//   softmax        two threads per query row (warps w and w + 4 reach the same TMEM lanes), each with
+//                  64 of the chunk's 128 keys: it reads its half row of S from TMEM, applies the
+//                  visibility rule (context / ancestor bitmask / prompt prefix), exchanges the
+//                  half-row maximum with its partner through shared memory, keeps the running
+//                  maximum and its half of the running sum (online softmax, log2 domain), writes
+//                  P = exp2(..) as bf16 into a K-major shared-memory tile and, when the maximum
+//                  moved, rescales its half of the row of the output accumulator in TMEM;
 //   O += P V       second UMMA chain, M = 128, N = D, K = 128 keys; the V chunk is used as it
 //                  lies in the cache ([key][D], i.e. MN-major for this product): the same staging
 //                  layout serves K (K-major for Q K^T) and V (MN-major for P V).
-// Roles: warps 0-3 softmax (TMEM lane group = warp), warp 4 issues the MMAs (one lane), warp 5
+// Roles: warps 0-7 softmax (TMEM lane group = warp % 4), warp 8 issues the MMAs (one lane), warp 9
 // brings Q and the K/V chunks in with TMA (two chunk buffers; box = 64 features x 128 rows, 128-byte
 // swizzle, no multicast) and clears the V rows past the last key before handing a chunk over.  Everything is handed over
 // through mbarriers with bounded waits; a wait that runs out raises the status word, the kernel
@@ -30,7 +32,8 @@ namespace bita {
 
 constexpr int AU_KEYS = 128;        // keys per chunk
 constexpr int AU_ROWS = 128;        // query rows per CTA
-constexpr int AU_THREADS = 192;
+constexpr int AU_THREADS = 320;      // 8 softmax warps, MMA warp, loader warp
+constexpr int AU_SOFTMAX = 256;      // softmax threads: two per query row
 constexpr int AU_ATOM = AU_ROWS * 128;   // bytes of one 128-row x 64-element swizzle atom column
 
 // MN-major operand (rows of the staged tile = K index, 64 elements of MN per 128-byte row):
@@ -133,6 +136,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   __shared__ __align__(8) uint64_t bar_cl_in, bar_cl_out;      // cluster merge: partials in / reads done
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
+  __shared__ float xchg[2][AU_ROWS];                // [half][row]: half-row maxima (and, at the end, sums)
 
   const int h = blockIdx.x, s = blockIdx.y;
   const int b = blockIdx.z / a.row_tiles, rt = blockIdx.z - b * a.row_tiles;
@@ -151,17 +155,17 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       mbar_init(smem_u32(&bar_v_full[i]), 1);
       mbar_init(smem_u32(&bar_v_empty[i]), 1);
       mbar_init(smem_u32(&bar_s_full[i]), 1);
-      mbar_init(smem_u32(&bar_s_free[i]), 128);
+      mbar_init(smem_u32(&bar_s_free[i]), AU_SOFTMAX);
     }
     mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_vfix), 1);
     mbar_init(smem_u32(&bar_cl_in), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_cl_out), (uint32_t)a.S);
-    mbar_init(smem_u32(&bar_p_full), 128);
+    mbar_init(smem_u32(&bar_p_full), AU_SOFTMAX);
     mbar_init(smem_u32(&bar_pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                  "r"(TMEM_COLS)
                  : "memory");
@@ -197,7 +201,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   const int fix = (n_cache % AU_KEYS != 0 && cache_chunks - 1 >= s && (cache_chunks - 1 - s) % a.S == 0)
                       ? (cache_chunks - 1 - s) / a.S : -1;
 
-  if (warp == 5) {
+  if (warp == 9) {
     // ---------------- loader (one lane issues; the warp clears the rows of the `fix` chunk)
     auto issue_tile = [&](int i, bool v_tile) {                  // lane 0 only
       const int ci = chunk_of(i);
@@ -268,7 +272,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     if (!ok) {
       for (int i = 0; i < 64; ++i) __nanosleep(1000);            // let the copies in flight land
     }
-  } else if (warp == 4) {
+  } else if (warp == 8) {
     // ---------------- MMA issuer
     if (lane == 0 && n > 0) {
       const uint32_t idesc_s = umma_idesc(AU_KEYS);                       // S: N = keys of a chunk
@@ -319,8 +323,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       }
     }
   } else {
-    // ---------------- softmax: thread r owns query row r of every row tile of the CTA
-    const int r = threadIdx.x;
+    // ---------------- softmax: threads r and r + 128 share query row r of every row tile of the
+    // CTA; thread half g takes keys [64 g, 64 g + 64) of a chunk and columns [g D/2, (g+1) D/2) of O
+    const int r = threadIdx.x & (AU_ROWS - 1), g = threadIdx.x >> 7;
+    constexpr int HK = AU_KEYS / 2, HD = D / 2;
     const float sc = a.scale_log2;
     int gr[RT];
     bool row_live[RT], sees_p[RT];
@@ -338,9 +344,9 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       }
       sees_p[t] = has_prompt && row_live[t] && a.sees_prompt[(size_t)b * a.sp_batch_stride + gr[t]] != 0;
       m_run[t] = -INFINITY;
-      l_run[t] = 0.f;
+      l_run[t] = 0.f;                                           // this thread's half of the row sum
     }
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     bool ok = true;
     for (int j = 0; j < n_steps; ++j) {
       const int i = j / RT;
@@ -352,23 +358,20 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       const bool live = second ? row_live[RT - 1] : row_live[0];
       const bool sp = second ? sees_p[RT - 1] : sees_p[0];
       const float m_old = second ? m_run[RT - 1] : m_run[0];
-      const uint32_t o_addr = lane_addr + COL_O + (second ? (uint32_t)((RT - 1) * D) : 0u);
-      const uint32_t r_row = (uint32_t)r;
+      const uint32_t o_addr = lane_addr + COL_O + (second ? (uint32_t)((RT - 1) * D) : 0u) + (uint32_t)(g * HD);
       const bool all_vis = !is_prompt && key0 + AU_KEYS <= C && live;
-      // Visibility of the chunk's 128 keys for this row as four 32-bit words: context keys are
-      // seen by every live row, block keys according to the row's ancestor bitmask (shifted to the
-      // key's place), prompt keys by mask rows only; keys past the last one by nobody.
-      uint32_t vm[4] = {0u, 0u, 0u, 0u};
+      // Visibility of this thread's 64 keys as two 32-bit words: context keys are seen by every
+      // live row, block keys according to the row's ancestor bitmask (shifted to the key's place),
+      // prompt keys by mask rows only; keys past the last one by nobody.
+      uint32_t vm[2] = {0u, 0u};
       if (live && !all_vis) {
-        if (is_prompt) {
 #pragma unroll
-          for (int w = 0; w < 4; ++w) {
+        for (int w2 = 0; w2 < 2; ++w2) {
+          const int w = 2 * g + w2;                             // word of the chunk
+          if (is_prompt) {
             const int nb = a.P - 32 * w;                        // prompt keys in this word
-            vm[w] = !sp || nb <= 0 ? 0u : (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u));
-          }
-        } else {
-#pragma unroll
-          for (int w = 0; w < 4; ++w) {
+            vm[w2] = !sp || nb <= 0 ? 0u : (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u));
+          } else {
             const int j0 = key0 + 32 * w - C;                   // block row index of the word's first key
             uint32_t word;
             if (j0 <= -32) {
@@ -385,30 +388,35 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
               }
               word = sh == 0 ? lo : __funnelshift_r(lo, hi, sh);
             }
-            vm[w] = word;
+            vm[w2] = word;
           }
         }
       }
       if (ok) ok = mbar_wait(smem_u32(&bar_s_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
-      const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(j & 1) * AU_KEYS;
-      // the whole row of scores into registers (one TMEM round trip); the buffer is free again
-      float sv[AU_KEYS];
-      tmem_ld128(s_addr, sv);
+      const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(j & 1) * AU_KEYS + (uint32_t)(g * HK);
+      // this thread's half row of scores into registers (one TMEM round trip); the buffer is free again
+      float sv[HK];
+      tmem_ld64(s_addr, sv);
       tc_fence_before();
       mbar_arrive_cta(smem_u32(&bar_s_free[j & 1]));
       float mx = -INFINITY;
       if (all_vis) {
 #pragma unroll
-        for (int e = 0; e < AU_KEYS; ++e) mx = fmaxf(mx, sv[e]);
+        for (int e = 0; e < HK; ++e) mx = fmaxf(mx, sv[e]);
       } else {
 #pragma unroll
-        for (int e = 0; e < AU_KEYS; ++e) {
+        for (int e = 0; e < HK; ++e) {
           if (!((vm[e >> 5] >> (e & 31)) & 1u)) sv[e] = -INFINITY;   // exp2(-inf) = 0 below
           mx = fmaxf(mx, sv[e]);
         }
       }
+      // the row maximum is the larger of the two halves': exchange through shared memory
+      xchg[g][r] = mx;
+      asm volatile("bar.sync 1, %0;" ::"n"(AU_SOFTMAX) : "memory");
+      mx = fmaxf(mx, xchg[g ^ 1][r]);
+      asm volatile("bar.sync 1, %0;" ::"n"(AU_SOFTMAX) : "memory");   // both have read: the slots may be rewritten
       const float m_new = fmaxf(m_old, mx * sc);
       const float sub = m_new == -INFINITY ? 0.f : m_new;
       const float corr = exp2f(m_old - sub);                    // 0 while nothing was seen before
@@ -416,10 +424,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       if (j > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
-      // P = exp2(s * scale - max), row sum, bf16 tile
+      // P = exp2(s * scale - max), half-row sum, bf16 tile (this thread's 64 keys are one swizzle atom)
       float sum = 0.f;
 #pragma unroll
-      for (int c0 = 0; c0 < AU_KEYS; c0 += 8) {
+      for (int c0 = 0; c0 < HK; c0 += 8) {
         uint32_t pk[4];
 #pragma unroll
         for (int e = 0; e < 8; e += 2) {
@@ -427,18 +435,18 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           sum += p0 + p1;
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off((int)r_row, c0 >> 3)), "r"(pk[0]),
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, g * 8 + (c0 >> 3))), "r"(pk[0]),
                      "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
                      : "memory");
       }
       if (i > 0 && __any_sync(0xffffffffu, corr != 1.0f)) {
         // the maximum of some row of this warp moved: bring the accumulator rows to their new
         // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch)
-        float ov[D];
-        if constexpr (D == 128) tmem_ld128(o_addr, ov); else tmem_ld64(o_addr, ov);
+        float ov[HD];
+        if constexpr (HD == 64) tmem_ld64(o_addr, ov); else tmem_ld32(o_addr, ov);
 #pragma unroll
-        for (int e = 0; e < D; ++e) ov[e] *= corr;
-        if constexpr (D == 128) tmem_st128(o_addr, ov); else tmem_st64(o_addr, ov);
+        for (int e = 0; e < HD; ++e) ov[e] *= corr;
+        if constexpr (HD == 64) tmem_st64(o_addr, ov); else tmem_st32(o_addr, ov);
       }
       if (second) { l_run[RT - 1] = l_run[RT - 1] * corr + sum; m_run[RT - 1] = m_new; }
       else { l_run[0] = l_run[0] * corr + sum; m_run[0] = m_new; }
@@ -450,22 +458,28 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     pdl_wait();
-    // ---- result of this slice: row r of O, per row tile
+    // ---- result of this slice: this thread's half of row r of O, per row tile
 #pragma unroll
     for (int t = 0; t < RT; ++t) {
-      float ov[D];
+      // the row sum is the sum of the two halves' (same reference maximum in both)
+      xchg[g][r] = l_run[t];
+      asm volatile("bar.sync 1, %0;" ::"n"(AU_SOFTMAX) : "memory");
+      const float l_row = l_run[t] + xchg[g ^ 1][r];
+      asm volatile("bar.sync 1, %0;" ::"n"(AU_SOFTMAX) : "memory");
+      float ov[HD];
+      const uint32_t o_addr = lane_addr + COL_O + (uint32_t)(t * D + g * HD);
       if (n_steps > 0 && ok) {
-        if constexpr (D == 128) tmem_ld128(lane_addr + COL_O + t * D, ov); else tmem_ld64(lane_addr + COL_O + t * D, ov);
+        if constexpr (HD == 64) tmem_ld64(o_addr, ov); else tmem_ld32(o_addr, ov);
       } else {
 #pragma unroll
-        for (int e = 0; e < D; ++e) ov[e] = 0.f;
+        for (int e = 0; e < HD; ++e) ov[e] = 0.f;
       }
       if (a.S == 1) {
-        const float inv = l_run[t] > 0.f ? 1.0f / l_run[t] : 0.f;
+        const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
         if (row_live[t]) {
-          bf16* dst = a.out + (((size_t)b * a.M + gr[t]) * a.H + h) * D;
+          bf16* dst = a.out + (((size_t)b * a.M + gr[t]) * a.H + h) * D + g * HD;
 #pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 8) {
+          for (int c0 = 0; c0 < HD; c0 += 8) {
             uint4 w;
             w.x = pack_bf16x2(ov[c0] * inv, ov[c0 + 1] * inv);     w.y = pack_bf16x2(ov[c0 + 2] * inv, ov[c0 + 3] * inv);
             w.z = pack_bf16x2(ov[c0 + 4] * inv, ov[c0 + 5] * inv); w.w = pack_bf16x2(ov[c0 + 6] * inv, ov[c0 + 7] * inv);
@@ -477,21 +491,23 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         // are free: every copy into them has landed and every MMA that read them is complete)
         if (row_live[t]) {
           const uint32_t prow = kv_s + (uint32_t)(t * AU_ROWS + r) * PSTRIDE;
-          asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(prow), "f"(m_run[t]), "f"(l_run[t]) : "memory");
+          if (g == 0) asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(prow), "f"(m_run[t]), "f"(l_row) : "memory");
 #pragma unroll
-          for (int e = 0; e < D; e += 4)
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(prow + 16 + e * 4), "f"(ov[e]), "f"(ov[e + 1]),
-                         "f"(ov[e + 2]), "f"(ov[e + 3])
+          for (int e = 0; e < HD; e += 4)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(prow + 16 + (g * HD + e) * 4), "f"(ov[e]),
+                         "f"(ov[e + 1]), "f"(ov[e + 2]), "f"(ov[e + 3])
                          : "memory");
         }
       } else {
         const size_t pbase = (((size_t)b * a.H + h) * a.S + s) * a.M;
         if (row_live[t]) {
-          a.part_ml[(pbase + gr[t]) * 2] = m_run[t];
-          a.part_ml[(pbase + gr[t]) * 2 + 1] = l_run[t];
-          float* dst = a.part_acc + (pbase + gr[t]) * D;
+          if (g == 0) {
+            a.part_ml[(pbase + gr[t]) * 2] = m_run[t];
+            a.part_ml[(pbase + gr[t]) * 2 + 1] = l_row;
+          }
+          float* dst = a.part_acc + (pbase + gr[t]) * D + g * HD;
 #pragma unroll
-          for (int e = 0; e < D; e += 4)
+          for (int e = 0; e < HD; e += 4)
             *reinterpret_cast<float4*>(dst + e) = make_float4(ov[e], ov[e + 1], ov[e + 2], ov[e + 3]);
         }
       }
@@ -573,7 +589,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
     mbar_wait_cluster(smem_u32(&bar_cl_out), 0, status);
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
