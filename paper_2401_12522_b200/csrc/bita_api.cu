@@ -542,8 +542,8 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
   if (!attr_set) {
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     attr_set = true;
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
