@@ -12,9 +12,8 @@
 //                  visibility rule (context / ancestor bitmask / prompt prefix), exchanges the
 //                  half-row maximum with its partner through shared memory, keeps the running
 //                  maximum and its half of the running sum (online softmax, log2 domain), writes
-//                  P = exp2(..) as bf16 into a K-major shared-memory tile (two of them alternate
-//                  when there is one row tile) and, when the maximum moved, rescales its half of
-//                  the row of the output accumulator in TMEM;
+//                  P = exp2(..) as bf16 into a K-major shared-memory tile and, when the maximum
+//                  moved, rescales its half of the row of the output accumulator in TMEM;
 //   O += P V       second UMMA chain, M = 128, N = D, K = 128 keys; the V chunk is used as it
 //                  lies in the cache ([key][D], i.e. MN-major for this product): the same staging
 //                  layout serves K (K-major for Q K^T) and V (MN-major for P V).
@@ -128,7 +127,6 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   constexpr uint32_t COL_S = 0, COL_O = 2 * AU_KEYS;   // two S buffers, then RT output accumulators of D columns
   static_assert(2 * AU_KEYS + RT * D <= 512, "tensor memory");
   constexpr uint32_t TMEM_COLS = 512;
-  constexpr int NP = RT == 1 ? 2 : 1;               // P tiles: two when shared memory allows (one row tile)
   constexpr uint32_t PSTRIDE = (D + 4) * 4;         // bytes of a partial row in shared memory: m, l, pad, O[D]
   extern __shared__ uint8_t smem_raw[];
   // K and V tiles of a chunk buffer are handed over separately: a K tile is free again once its
@@ -136,7 +134,6 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   __shared__ __align__(8) uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
   __shared__ __align__(8) uint64_t bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done, bar_q, bar_vfix;
   __shared__ __align__(8) uint64_t bar_cl_in, bar_cl_out;      // cluster merge: partials in / reads done
-  __shared__ __align__(8) uint64_t bar_p_free[2];              // P tile read by its P V product
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
   __shared__ float xchg[2][AU_ROWS];                // [half][row]: half-row maxima (and, at the end, sums)
@@ -162,8 +159,6 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
     mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_vfix), 1);
-    mbar_init(smem_u32(&bar_p_free[0]), 1);
-    mbar_init(smem_u32(&bar_p_free[1]), 1);
     mbar_init(smem_u32(&bar_cl_in), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_cl_out), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_p_full), AU_SOFTMAX);
@@ -319,11 +314,10 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
 #pragma unroll
         for (int kk = 0; kk < AU_KEYS / 16; ++kk) {
-          const uint64_t da = umma_smem_desc(p_s + (j % NP) * 2 * AU_ATOM + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
+          const uint64_t da = umma_smem_desc(p_s + (kk >> 2) * AU_ATOM) + (uint64_t)(2 * (kk & 3));
           const uint64_t db = umma_smem_desc_mn(vs + kk * 16 * 128, AU_ATOM);
           umma_bf16(tmem + COL_O + (uint32_t)(t * D), da, db, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bar_p_free[j % NP]));
         if (t == RT - 1) umma_commit(smem_u32(&bar_v_empty[i & 1]));
         umma_commit(smem_u32(&bar_pv_done));
       }
@@ -426,8 +420,8 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       const float m_new = fmaxf(m_old, mx * sc);
       const float sub = m_new == -INFINITY ? 0.f : m_new;
       const float corr = exp2f(m_old - sub);                    // 0 while nothing was seen before
-      // P goes into tile j % NP, which the P V product of step j - NP read
-      if (j >= NP && ok) ok = mbar_wait(smem_u32(&bar_p_free[j % NP]), ((uint32_t)(j / NP) & 1u) ^ 1u, status);
+      // P overwrites the tile the previous P V product reads, and the rescale touches an accumulator
+      if (j > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       // P = exp2(s * scale - max), half-row sum, bf16 tile (this thread's 64 keys are one swizzle atom)
@@ -441,17 +435,13 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           sum += p0 + p1;
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + (j % NP) * 2 * AU_ATOM + au_off(r, g * 8 + (c0 >> 3))), "r"(pk[0]),
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_s + au_off(r, g * 8 + (c0 >> 3))), "r"(pk[0]),
                      "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
                      : "memory");
       }
       if (i > 0 && __any_sync(0xffffffffu, corr != 1.0f)) {
         // the maximum of some row of this warp moved: bring the accumulator rows to their new
-        // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch), once
-        // the P V product of the step before has left the accumulator alone
-        if (ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
+        // reference (the TMEM instructions are warp-wide, so the whole warp takes the branch)
         float ov[HD];
         if constexpr (HD == 64) tmem_ld64(o_addr, ov); else tmem_ld32(o_addr, ov);
 #pragma unroll

@@ -537,11 +537,11 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)a.D);
   const int RT = a.M > AU_ROWS ? 2 : 1;                          // row tiles per CTA
   const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
-  const size_t smem = (RT + 4) * tile + (RT == 1 ? 2 : 1) * 2 * AU_ATOM + 1024;   // Q (RT tiles), 2 x (K, V), P tile(s)
+  const size_t smem = (RT + 4) * tile + 2 * AU_ATOM + 1024;       // Q (RT tiles), 2 x (K, V), P
   static bool attr_set = false;
   if (!attr_set) {
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     attr_set = true;
