@@ -83,7 +83,7 @@ def test_tree_attention_matches_oracle(B, N, H, H_kv, D, P, C):
 
 # ------------------------------------------------------------------ the whole pass, lockstep
 
-@pytest.mark.parametrize("plen", [140, 300])
+@pytest.mark.parametrize("plen", [1, 140, 300])
 def test_first_pass_in_several_blocks(plen):
     """Prompts longer than one block of the first pass (248 query rows): 140 tokens make one block of
     143 rows (past 128: two attention row tiles), 300 make two blocks of 150."""
@@ -111,6 +111,7 @@ TEMPLATES = {
     "comb-n3k5-pernode": (lambda: synth.comb_template(3, 5), 3),
     "comb-n4k3-pernode": (lambda: synth.comb_template(4, 3), 4),
     "comb-n4k5-pernode": (lambda: synth.comb_template(4, 5), 4),     # 105 rows: past 96, one row tile
+    "comb-n4k12-pernode": (lambda: synth.comb_template(4, 12), 4),   # 245 rows: near the limit, two row tiles
     "chain": (lambda: synth.chain_template(3), 3),
     "empty": (lambda: synth.empty_template(), 3),
     "product-pernode": (lambda: synth.product_rule_template((3, 3, 3), (3, 3, 3), per_node_groups=True), 3),
