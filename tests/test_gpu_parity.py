@@ -180,6 +180,48 @@ def test_gpu_generation_is_lossless_against_its_own_autoregressive_run():
         assert top[0] - top[1] <= LOGIT_TOL_RMS * rms, f"sequences diverge at {first} with a clear margin"
 
 
+def test_full_depth_7b_generation_is_lossless_against_its_own_autoregressive_run():
+    """The measured 7B configuration at its full depth (32 layers, 64-node tree, 69 rows): the BiTA
+    loop with planted drafts and the one-token-per-pass loop of the library emit the same tokens.
+    No oracle at this size: where the two diverge, the library's own top-1 / top-2 margin at that
+    position must be below the logit tolerance (a property that holds at any size)."""
+    from paper_2401_12522_b200 import Bita
+    shape = synth.CONFIGS["7b"]
+    seed = 0x5EED0004
+    w = synth.make_weights(shape, seed, dtype=torch.bfloat16, device="cuda:0")
+    prompt = prompt_tokens(seed, 96, shape.V)
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    n_new = 14
+    ar = Bita(shape, w, synth.empty_template(), C_max=256)
+    ar.enable_debug(True)
+    seq_ar = list(ar.prefill(prompt)["out_tokens"])
+    margins = [None]                                           # margin behind token i of the run (None: first pass)
+    while len(seq_ar) < n_new:
+        seq_ar += ar.step()["out_tokens"]
+        row = ar.debug_logits(1)[0].float()
+        top = torch.topk(row, 2).values
+        margins.append(float(top[0] - top[1]) / float(row.pow(2).mean().sqrt()))
+    ar.close()
+    bt = Bita(shape, w, tmpl, C_max=256)
+    seq = list(bt.prefill(prompt)["out_tokens"])
+    step, passes = 0, 0
+    while len(seq) < n_new:
+        done = len(seq)
+        tree = synth.plant_tree(tmpl, [-1] * tmpl.N, seq_ar[done: done + 4], seed, step, 0.7, shape.V)
+        rec = bt.step(tree)
+        assert 1 <= rec["n_out"] <= 5
+        seq += rec["out_tokens"]
+        step += 1
+        passes += 1
+    bt.close()
+    assert passes < n_new - 1                                  # planted paths were accepted: fewer passes than tokens
+    seq, seq_ar = seq[:n_new], seq_ar[:n_new]
+    if seq != seq_ar:
+        first = next(i for i in range(n_new) if seq[i] != seq_ar[i])
+        assert margins[first] is not None and margins[first] <= LOGIT_TOL_RMS * 2, \
+            f"sequences diverge at {first} although the margin there is {margins[first]:.3f} x RMS"
+
+
 def test_step_after_reset_reproduces_the_first_run():
     from paper_2401_12522_b200 import Bita
     shape = synth.CONFIGS["tiny"]
