@@ -1,9 +1,10 @@
 // Tree-based attention (Sec. 3.2, Fig. 6) on the tcgen05 tensor cores.
 //
 // One CTA = one query head x one key slice x RT row tiles of 128 query rows (RT = 2 for blocks of
-// more than 128 rows, so that both tiles share every K/V chunk that is read; arguments, slicing and the
-// partial-result format: attention_common.cuh).  The slice's keys are walked in chunks of 128; the
-// cache chunks come first, the prompt-prefix chunk last; slice s takes chunks s, s + S, ...:
+// more than 128 rows, so that both tiles share every K/V chunk that is read; arguments, slicing
+// and the partial-result format: attention_common.cuh).  Keys are walked in chunks of 128, the
+// cache chunks first, the prompt-prefix chunk last; slice s takes chunks s, s + S, ...  Per chunk
+// and row tile:
 //   S = Q K^T      one UMMA chain, M = 128 (query rows), N = 128 (keys), K = D; Q and the K chunk
 //                  sit in shared memory as K-major 128-byte-swizzled tiles; S lands in TMEM with
 //                  lane = query row, column = key (two S buffers alternate);
@@ -19,9 +20,9 @@
 //                  layout serves K (K-major for Q K^T) and V (MN-major for P V).
 // Roles: warps 0-7 softmax (TMEM lane group = warp % 4), warp 8 issues the MMAs (one lane), warp 9
 // brings Q and the K/V chunks in with TMA (two chunk buffers; box = 64 features x 128 rows, 128-byte
-// swizzle, no multicast) and clears the V rows past the last key before handing a chunk over.  Everything is handed over
-// through mbarriers with bounded waits; a wait that runs out raises the status word, the kernel
-// drains and frees its TMEM.  Several key slices of one (sequence, head, row tile) run as one
+// swizzle, no multicast) and clears the V rows past the last key before handing a chunk over.
+// Everything is handed over through mbarriers with bounded waits; a wait that runs out raises the
+// status word, the kernel drains and frees its TMEM.  Several key slices of one (sequence, head, row tile) run as one
 // thread-block cluster and merge their partial results through distributed shared memory.
 #pragma once
 
@@ -31,7 +32,7 @@
 namespace bita {
 
 constexpr int AU_KEYS = 128;        // keys per chunk
-constexpr int AU_ROWS = 128;        // query rows per CTA
+constexpr int AU_ROWS = 128;        // query rows per row tile
 constexpr int AU_THREADS = 320;      // 8 softmax warps, MMA warp, loader warp
 constexpr int AU_SOFTMAX = 256;      // softmax threads: two per query row
 constexpr int AU_ATOM = AU_ROWS * 128;   // bytes of one 128-row x 64-element swizzle atom column
