@@ -315,8 +315,11 @@ def run_ours(args, shape, tmpl):
     t0 = time.perf_counter()
     e0.record()
     got = 0
+    step_wall = []
     for s in range(W, total_steps):
+        t_s = time.perf_counter()
         got += ctx.step(trees[s])["n_out"]
+        step_wall.append((time.perf_counter() - t_s) * 1e3)
     e1.record()
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
@@ -354,6 +357,7 @@ def run_ours(args, shape, tmpl):
             "config": {"workload": _workload_name(shape, tmpl, args.planted), "l2": "inputs (weights) larger than L2",
                        "tokens_per_step": tokens_timed / K, "parallelism": f"replicas x{world}"},
             "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
+                    "p50_ms": statistics.median(step_wall), "p90_ms": sorted(step_wall)[int(0.9 * (len(step_wall) - 1))],
                     "h2d_bytes_per_step": 4 * tmpl.N, "d2h_bytes_per_step": 4 * (5 + 2 * 16 + 1 + 160)},
             "gpu_launches": launches,
             "clocks": clocks,
