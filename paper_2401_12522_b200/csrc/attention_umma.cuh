@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   // Q K^T chain is done (long before the chunk's P V product), so the next K is on its way early.
   __shared__ __align__(8) uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
   __shared__ __align__(8) uint64_t bar_s_full[2], bar_s_free[2], bar_p_full, bar_pv_done, bar_q, bar_vfix;
-  __shared__ __align__(8) uint64_t bar_cl_in[8], bar_cl_out;   // cluster merge: slice p's partials in / reads done
+  __shared__ __align__(8) uint64_t bar_cl_in, bar_cl_out;      // cluster merge: partials in / reads done
   __shared__ uint32_t tmem_slot;
   __shared__ int32_t status_local;                  // stands in when the caller gave no status word
   __shared__ float xchg[2][AU_ROWS];                // [half][row]: half-row maxima (and, at the end, sums)
@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     }
     mbar_init(smem_u32(&bar_q), 1);
     mbar_init(smem_u32(&bar_vfix), 1);
-    for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bar_cl_in[i]), 1);
+    mbar_init(smem_u32(&bar_cl_in), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_cl_out), (uint32_t)a.S);
     mbar_init(smem_u32(&bar_p_full), AU_SOFTMAX);
     mbar_init(smem_u32(&bar_pv_done), 1);
@@ -517,20 +517,18 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   }
 
   // ---- merge inside the cluster: the S slices of this (sequence, head, row tile) are the CTAs of
-  // one cluster (rank = slice).  Each leaves its partial rows in its own shared memory and tells every
-  // peer (one mbarrier per slice in every CTA); each CTA merges an equal share of the rows, reading the
-  // slices' partials through distributed shared memory as they come in - the slice that holds the
-  // block's last keys, the last to finish, is asked last - and combining them in that fixed order.
-  // A second round of arrivals keeps every CTA alive until its peers have finished reading it.
-  // All waits are bounded mbarrier waits.
+  // one cluster (rank = slice).  Each leaves its partial rows in its own shared memory, tells every
+  // peer, and once all S are in merges an equal share of the rows, reading the peers' partials
+  // through distributed shared memory, in slice order.  A second round of arrivals keeps every CTA
+  // alive until its peers have finished reading it.  Both waits are bounded mbarrier waits.
   tc_fence_before();
   __syncthreads();
   if (a.S > 1 && a.cluster) {
     if (threadIdx.x == 0) {
       asm volatile("fence.acq_rel.cluster;" ::: "memory");
-      for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_in[s]), (uint32_t)p));
+      for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_in), (uint32_t)p));
     }
-    const int s_late = (cache_chunks - 1) % a.S;                // the slice with the last cache chunk
+    mbar_wait_cluster(smem_u32(&bar_cl_in), 0, status);
     constexpr int VW = D / 32;
     const int rows_here = min(RT * AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
@@ -538,18 +536,16 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     for (int r0 = r_lo + warp; r0 < r_hi; r0 += NW * RR) {
       float ms[RR][8], ls[RR][8], v[RR][8][VW];
 #pragma unroll
-      for (int p = 0; p < 8; ++p) {                             // slot p holds slice (s_late + 1 + p) mod S
-        const int peer = p < a.S ? (s_late + 1 + p) % a.S : 0;
-        if (p < a.S) mbar_wait_cluster(smem_u32(&bar_cl_in[peer]), 0, status);
+      for (int u = 0; u < RR; ++u) {
+        const int r = min(r0 + u * NW, r_hi - 1);               // clamped: surplus slots redo the last row
 #pragma unroll
-        for (int u = 0; u < RR; ++u) {
-          const int r = min(r0 + u * NW, r_hi - 1);             // clamped: surplus slots redo the last row
+        for (int p = 0; p < 8; ++p) {
           ms[u][p] = -INFINITY;
           ls[u][p] = 0.f;
 #pragma unroll
           for (int e = 0; e < VW; ++e) v[u][p][e] = 0.f;
           if (p < a.S) {
-            const uint32_t prow = mapa_u32(kv_s + (uint32_t)r * PSTRIDE, (uint32_t)peer);
+            const uint32_t prow = mapa_u32(kv_s + (uint32_t)r * PSTRIDE, (uint32_t)p);
             const float2 ml = ld_dsmem_f2(prow);
             ms[u][p] = ml.x;
             ls[u][p] = ml.y;
