@@ -219,6 +219,101 @@ def test_fig3_emitted_per_pass_pattern():
     assert orc.next_tree(blk, np.array([[[31], [32], [33]]]), cur) == [33, -1, -1]
 
 
+def _gold_cases(name):
+    """(header dict, [(case fields, expected tree)]) of a next-tree golden file."""
+    rows = _read_gold(name)
+    head = {r[0]: int(r[1]) for r in rows if r[0] in ("n", "k")}
+    cases, cur = [], None
+    for r in rows:
+        if r[0] == "case":
+            cur = {r[i]: int(r[i + 1]) for i in range(1, len(r), 2)}
+        elif r[0] == "tree":
+            cases.append((cur, [int(v) for v in r[1:]]))
+    return head, cases
+
+
+def test_next_tree_takes_the_group_of_the_last_accepted_node_alg1_golden():
+    """Algorithm 1, last step of each branch, on the Fig. 4 tree with a mask group per node: the
+    expected trees were written out by hand in the golden file; every scripted prediction is a
+    distinct id, so a wrong group, a swapped mask/candidate index or a shifted depth changes a token."""
+    head, cases = _gold_cases("alg1_next_tree_comb_n4k3.txt")
+    n, k = head["n"], head["k"]
+    blk = block_for(synth.comb_template(n, k), n)
+    assert blk.G == n * k + 1
+    topk = np.zeros((blk.G, n, k), dtype=np.int64)
+    for g, at in enumerate(blk.attach):
+        for r in range(1, n + 1):
+            for j in range(1, k + 1):
+                topk[g, r - 1, j - 1] = 100 * (at + 1) + 10 * r + j
+    assert len(set(topk.ravel().tolist())) == topk.size
+    assert len(cases) == 5
+    for case, want in cases:
+        assert orc.next_tree(blk, topk, case["last"]) == want
+    # the same through the walk: accepting exactly the path to `last` selects that group
+    for case, want in cases:
+        path, x = [], case["last"]
+        while x >= 0:
+            path.append(x)
+            x = blk.parent[x]
+        path.reverse()
+        tree = list(range(500, 500 + blk.N))                    # distinct draft tokens
+        am = [499] * (1 + blk.N)                                # predictions that match nothing ...
+        prev = -1
+        for x in path:                                          # ... except along the path
+            am[1 + prev] = tree[x]
+            prev = x
+        acc, out, cur = orc.verify_walk(blk, tree, am)
+        assert acc == path and cur == case["last"]
+        assert orc.next_tree(blk, topk, cur) == want
+
+
+def test_next_tree_single_group_drops_the_first_c_masks_fig3_golden():
+    """One mask group after the last token and k > 1 candidates per mask: after c accepted drafts
+    depth r of the next tree holds the candidates of mask c + r (Fig. 3 caption), by hand in the
+    golden file."""
+    head, cases = _gold_cases("fig3_single_group_shift.txt")
+    n, k = head["n"], head["k"]
+    blk = block_for(synth.comb_template(n, k, per_node_groups=False), n)
+    assert blk.G == 1
+    topk = np.array([[[10 * r + j for j in range(1, k + 1)] for r in range(1, n + 1)]])
+    assert len(cases) == 6
+    for case, want in cases:
+        assert blk.depth[case["last"]] == case["c"] if case["last"] >= 0 else case["c"] == 0
+        assert orc.next_tree(blk, topk, case["last"]) == want
+
+
+def test_first_pass_drafts_the_top_k_of_each_mask_alg1_t1():
+    """Algorithm 1, t = 1: the last query token's top-1 is emitted and C^1 holds the top k of each
+    mask token.  A scripted model (one layer whose attention and FFN add nothing, mask embedding i
+    = unit vector 1 + i, LM-head column 1 + i = the scores of mask i) makes the logits of every
+    mask row known in advance; the expected tree is the c = 0 case of the hand-written golden."""
+    head, cases = _gold_cases("fig3_single_group_shift.txt")
+    n, k = head["n"], head["k"]
+    want = [t for c, t in cases if c["c"] == 0][0]
+    d, V = 8, 64
+    lm = np.zeros((V, d))
+    lm[7, 0] = 1.0                                              # every query token embeds to e_0: its argmax is 7
+    for r in range(1, n + 1):
+        for j in range(1, k + 1):
+            lm[10 * r + j, r] = 4.0 - j                         # mask r: candidate j has the j-th largest score
+    z = lambda *s: np.zeros(s)
+    layer = dict(wqkv=z(3 * d, d), wo=z(d, d), wg=z(8, d), wu=z(8, d), wd=z(d, 8), g_attn=np.ones(d),
+                 g_ffn=np.ones(d), prompt_k=z(1, 0, d), prompt_v=z(1, 0, d))
+    tok = z(V, d)
+    tok[:, 0] = 1.0
+    me = z(n, d)
+    for i in range(n):
+        me[i, 1 + i] = 1.0
+    m = orc.Model(L=1, d=d, H=1, H_kv=1, D=d, F=8, V=V, P=0, n_mask=n, rms_eps=1e-5, rope_theta=1e4,
+                  weights=dict(tok_emb=tok, mask_emb=me, g_final=np.ones(d), lm_head=lm, layers=[layer]))
+    for tmpl in (synth.comb_template(n, k), synth.comb_template(n, k, per_node_groups=False)):
+        blk = block_for(tmpl, n)
+        st = orc.State(m)
+        rec = orc.prefill(m, blk, st, [3, 1, 4, 1, 5])
+        assert rec["out_tokens"] == [7] and rec["n_out"] == 1
+        assert rec["next_tree"] == want and st.tree == want and st.root == 7 and st.C == 5
+
+
 def _algorithm1_flat_walk(n, k, cand, logits_argmax):
     """Independent restatement of the paper's verification for its comb tree, on flattened row indices.
 
