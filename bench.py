@@ -121,43 +121,84 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-# reference arm: the CPU oracle as it stands, on a bounded sample of the same workload
-def _oracle_sample(shape, tmpl, n_steps, n_warm, fraction):
-    """Times `n_steps` oracle samples; a sample is ONE decoder layer of the step's packed block.
+# CPU oracle legs: `cpu_baseline` of our arm and the whole of `--impl reference`
+def _seeded_state(orc, model, shape, C):
+    """Oracle decoding state with C cached tokens of seeded random keys/values (the time of a pass
+    does not depend on their values) and an arbitrary last token."""
+    st = orc.State(model)
+    for l in range(shape.L):
+        st.k[l] = synth.pseudo_normal(PROMPT_SEED, 1000 + 2 * l, (shape.H_kv, C, shape.D), 1.0).double().numpy()
+        st.v[l] = synth.pseudo_normal(PROMPT_SEED, 1001 + 2 * l, (shape.H_kv, C, shape.D), 1.0).double().numpy()
+    st.root = 1
+    return st
 
-    The full-step time is estimated as L x (layer time) + (final norm + LM head + selection + walk),
-    the latter measured once.  Returns (tokens/s, ms per estimated full step, description, cores).
-    """
-    import numpy as np
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from helpers import block_for, oracle_model  # noqa
+
+def _gen_device():
+    return "cuda:0" if torch.cuda.is_available() else "cpu"
+
+
+def oracle_whole_steps(shape, tmpl, n_steps, n_warm, fraction):
+    """Times whole oracle passes (`orc.bita_step`: pack, every layer, LM head, selection, walk, next
+    tree, cache append) of the workload's block, the oracle exactly as the tests call it.
+    Returns (tokens/s, ms per pass, description, cores)."""
     from oracle import bita_oracle as orc
+    from oracle.inputs import block_for, oracle_model
+    cores = len(os.sched_getaffinity(0))
+    torch.set_num_threads(cores)
+    # the model's weights as fp32 host arrays, generated off the clock (on the GPU when there is one)
+    weights = synth.make_weights(shape, MODEL_SEED, dtype=torch.bfloat16, device=_gen_device())
+    model = oracle_model(shape, MODEL_SEED, weights=weights)
+    del weights
+    if torch.cuda.is_available():
+        torch.cuda.empty_cache()
+    blk = block_for(tmpl, shape.n_mask)
+    st = _seeded_state(orc, model, shape, shape.prompt_len)
+    tree = synth.uniform_ints(PLANT_SEED, 77, blk.N, shape.V).tolist()
+    times = []
+    for i in range(n_warm + n_steps):
+        t0 = time.perf_counter()
+        rec = orc.bita_step(model, blk, st, tree)
+        times.append(time.perf_counter() - t0)
+        tree = rec["next_tree"]
+    ms = 1e3 * sum(times[n_warm:]) / max(1, n_steps)
+    tps = _expected_tokens_per_step(tmpl, fraction) / (ms * 1e-3)
+    desc = (f"{n_steps} whole oracle passes (orc.bita_step, all {shape.L} layers + LM head + selection + walk) of the "
+            f"{shape.name} block ({blk.M} rows) on a cache of {shape.prompt_len} seeded random tokens; fp64 numpy; "
+            f"tokens per pass = expectation of the planting recipe")
+    return tps, ms, desc, cores
 
+
+def oracle_layer_samples(shape, tmpl, n_steps, n_warm, fraction):
+    """For models whose whole oracle pass takes minutes (70B): a sample is ONE decoder layer of the
+    pass; the whole pass is ESTIMATED as L x (mean layer time) + (LM head + selection + walk, timed once).
+    Returns (tokens/s of the estimate, ms per sample, ms per estimated pass, description, cores)."""
+    import numpy as np
+    from oracle import bita_oracle as orc
+    from oracle.inputs import block_for, oracle_model
     cores = len(os.sched_getaffinity(0))
     torch.set_num_threads(cores)
     one = shape.with_layers(1)
-    model = oracle_model(one, MODEL_SEED)
-    # fp64 copies of the sampled layer, so that a sample times the arithmetic and not the conversion
-    model.w["layers"][0] = {k: np.asarray(v, dtype=np.float64) for k, v in model.w["layers"][0].items()}
-    lm64 = np.asarray(model.w["lm_head"], dtype=np.float64)
+    weights = synth.make_weights(one, MODEL_SEED, dtype=torch.bfloat16, device=_gen_device())
+    model = oracle_model(one, MODEL_SEED, weights=weights)
+    del weights
+    if torch.cuda.is_available():
+        torch.cuda.empty_cache()
     blk = block_for(tmpl, shape.n_mask)
-    C = shape.prompt_len
-    rng_k = synth.pseudo_normal(PROMPT_SEED, 31, (shape.H_kv, C, shape.D), 1.0).double().numpy()
-    rng_v = synth.pseudo_normal(PROMPT_SEED, 32, (shape.H_kv, C, shape.D), 1.0).double().numpy()
+    st = _seeded_state(orc, model, one, shape.prompt_len)
     x = synth.pseudo_normal(PROMPT_SEED, 33, (blk.M, shape.d), 1.0).double().numpy()
-    pos = C + blk.rel_pos
+    pos = shape.prompt_len + blk.rel_pos
 
     def layer():
-        return orc._layer(model, model.w["layers"][0], x, pos, rng_k, rng_v, blk.vis, blk.sees_prompt)
+        return orc._layer(model, model.w["layers"][0], x, pos, st.k[0], st.v[0], blk.vis, blk.sees_prompt)
 
     def head():
-        logits = orc.rmsnorm(x, model.w["g_final"], model.rms_eps) @ lm64.T
+        logits = orc.rmsnorm(x, model.w["g_final"], model.rms_eps) @ np.asarray(model.w["lm_head"], dtype=np.float64).T
         am = [orc.argmax_lowest(logits[r]) for r in range(1 + blk.N)]
         tk = np.zeros((blk.G, blk.n, blk.k_max), dtype=np.int64)
         for g in range(blk.G):
             for i in range(blk.n):
                 tk[g, i], _ = orc.topk_sorted(logits[blk.mask_row(g, i)], blk.k_max)
-        acc, out, cur = orc.verify_walk(blk, [1] * blk.N, am)
+        _, _, cur = orc.verify_walk(blk, [1] * blk.N, am)
         orc.next_tree(blk, tk, cur)
 
     t0 = time.perf_counter()
@@ -171,24 +212,48 @@ def _oracle_sample(shape, tmpl, n_steps, n_warm, fraction):
     t_layer = (time.perf_counter() - t0) / max(1, n_steps)
     full = shape.L * t_layer + t_head
     tps = _expected_tokens_per_step(tmpl, fraction) / full
-    desc = (f"{n_steps} samples of one decoder layer of the {shape.name} step ({blk.M} rows, random KV context of "
-            f"{C} tokens, weights held in fp64), scaled x{shape.L} layers + LM head/selection/walk measured once; "
-            f"tokens per step = expectation of the planting recipe")
-    return tps, full * 1e3, desc, cores
+    desc = (f"ESTIMATE: {n_steps} samples of one decoder layer of the {shape.name} pass ({blk.M} rows, cache of "
+            f"{shape.prompt_len} seeded random tokens; orc._layer as it stands), scaled x{shape.L} layers + LM head / "
+            f"selection / walk timed once ({t_head * 1e3:.0f} ms); a whole fp64 pass of this model takes minutes; "
+            f"tokens per pass = expectation of the planting recipe")
+    return tps, t_layer * 1e3, full * 1e3, desc, cores
+
+
+def oracle_leg(shape, tmpl, n_steps, n_warm, fraction, whole_steps=None):
+    """cpu_baseline record of a workload: whole passes where one takes seconds, the labelled
+    layer-sample estimate where it takes minutes."""
+    if shape.streamed_params > 20e9:
+        tps, ms_sample, ms_full, desc, cores = oracle_layer_samples(shape, tmpl, n_steps, n_warm, fraction)
+        return {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                "ms_per_step": ms_full, "ms_per_sample": ms_sample, "estimated": True}
+    tps, ms, desc, cores = oracle_whole_steps(shape, tmpl, n_steps if whole_steps is None else whole_steps, n_warm,
+                                              fraction)
+    return {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "ms_per_step": ms,
+            "ms_per_sample": ms, "estimated": False}
+
+
+def _config(shape, tmpl, fraction, world):
+    """The `config` object, identical in our arm and in the reference arm."""
+    return {"workload": _workload_name(shape, tmpl, fraction), "l2": "inputs (weights) larger than L2",
+            "tokens_per_step_expected": _expected_tokens_per_step(tmpl, fraction),
+            "parallelism": f"replicas x{world}"}
 
 
 def run_reference(args, shape, tmpl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    tps, ms, desc, cores = _oracle_sample(shape, tmpl, args.steps, args.warmup, args.planted)
+    leg = oracle_leg(shape, tmpl, args.steps, args.warmup, args.planted)
+    # `ms_per_step` is the wall time of one timed sample, so that steps x ms_per_step is the timed
+    # region of this run; for the 70B shape the sample is one layer and `value` the labelled estimate
     line = {
-        "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic",
-        "config": {"workload": _workload_name(shape, tmpl, args.planted)},
-        "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
-        "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "impl": "reference", "metric": METRIC, "value": leg["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": leg["ms_per_sample"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config(shape, tmpl, args.planted, max(1, args.gpus)),
+        "cpu_baseline": {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample", "estimated")},
+        "estimated_full_step_ms": leg["ms_per_step"],
+        "e2e": {"value": leg["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
@@ -248,22 +313,11 @@ def aggregate_over_ranks(dist_mod, world: int, dev_ms: float, e2e_ms: float, tok
     return dev_ms, e2e_ms, float(toks[0])
 
 
-def run_ours(args, shape, tmpl):
+def measure_workload(shape, tmpl, K, W, fraction, rank, world, local, dist):
+    """All device-side measurements of one workload on this rank's GPU.  Returns a dict of raw numbers
+    (times are this rank's; `aggregate_over_ranks` combines them)."""
     from paper_2401_12522_b200 import Bita
-    from paper_2401_12522_b200.build import build
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    if rank == 0:
-        build()
-    if world > 1:
-        dist.barrier()
     dev = torch.device(f"cuda:{local}")
-    torch.cuda.set_device(dev)
-    K, W = args.steps, args.warmup
     total_steps = K + W
     depth = max(tmpl.depths(), default=0)
     rows = 1 + tmpl.N + tmpl.G * shape.n_mask
@@ -273,20 +327,20 @@ def run_ours(args, shape, tmpl):
     prompt = synth.uniform_ints(replica_plan(rank, shape)["prompt_seed"], 5001, shape.prompt_len, shape.V).tolist()
     ctx = Bita(shape, weights, tmpl, C_max=C_max, device=dev)
 
-    def start():
-        ctx.reset()
-        r = ctx.prefill(prompt)
-        ctx._len, ctx._root, ctx._tree = r["new_len"], r["out_tokens"][-1], r["next_tree"]
-
-    start()
-    trees, emitted = build_trees(ctx, shape, tmpl, total_steps, args.planted)
-    trees_dev = torch.tensor(trees, dtype=torch.int32, device=dev) if tmpl.N else None
-    tokens_timed = sum(emitted[W:])
+    def start(c=ctx):
+        c.reset()
+        r = c.prefill(prompt)
+        c._len, c._root, c._tree = r["new_len"], r["out_tokens"][-1], r["next_tree"]
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(dev)
+
+    start()
+    trees, emitted = build_trees(ctx, shape, tmpl, total_steps, fraction)
+    trees_dev = torch.tensor(trees, dtype=torch.int32, device=dev) if tmpl.N else None
+    tokens_timed = sum(emitted[W:])
 
     # ---- device-resident timing: inputs already in HBM, no host sync inside the timed region
     start()
@@ -325,7 +379,8 @@ def run_ours(args, shape, tmpl):
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
     assert got == tokens_timed
 
-    # ---- per-kernel timing pass for the roofline (events around every projection / attention launch)
+    # ---- per-family timing pass for the roofline: one CUDA event on the library's stream wherever the
+    # kernel family changes (runs of consecutive projections are timed as they overlap in a normal pass)
     start()
     ctx.set_kernel_timing(True)
     fam_ms, fam_n = [0.0, 0.0], [0, 0]
@@ -337,43 +392,109 @@ def run_ours(args, shape, tmpl):
         fam_n = [a + b for a, b in zip(fam_n, n)]
     ctx.set_kernel_timing(False)
     ctx.step_finish()
-
-    dev_ms, e2e_ms, total_tokens = aggregate_over_ranks(dist if world > 1 else None, world, dev_ms, e2e_ms,
-                                                        tokens_timed, dev)
-
-    if rank == 0:
-        peak, peak_src = _peaks()
-        weight_bytes = shape.streamed_params * 2
-        gemm_ms = fam_ms[0] / max(1, fam_n[0])                    # average projection launch
-        gemm_bytes = weight_bytes / (fam_n[0] / n_prof)            # algorithmic bytes of an average launch
-        achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
-        mean_C = shape.prompt_len + sum(emitted[:W]) + sum(emitted[W:]) / 2
-        step_bytes = weight_bytes + shape.kv_bytes_per_token() * mean_C
-        step_ms = dev_ms / K
-        line = {
-            "metric": METRIC, "value": total_tokens / (dev_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": _workload_name(shape, tmpl, args.planted), "l2": "inputs (weights) larger than L2",
-                       "tokens_per_step": tokens_timed / K, "parallelism": f"replicas x{world}"},
-            "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
-                    "p50_ms": statistics.median(step_wall), "p90_ms": sorted(step_wall)[int(0.9 * (len(step_wall) - 1))],
-                    "h2d_bytes_per_step": 4 * tmpl.N, "d2h_bytes_per_step": 4 * (5 + 2 * 16 + 1 + 160)},
-            "gpu_launches": launches,
-            "clocks": clocks,
-            "step_hbm_frac": (step_bytes / (step_ms * 1e-3) / 1e9) / peak,
-            "roofline": {"bound": "hbm", "kernel": "projection (weight-streaming GEMM), mean over the step's launches; events at the boundaries of runs of consecutive projections",
-                         "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-                         "frac": achieved / peak, "algorithmic_bytes_per_launch": gemm_bytes,
-                         "traffic": _traffic_per_mean_launch(shape, tmpl),
-                         "attention_ms_per_step": fam_ms[1] / n_prof, "projection_ms_per_step": fam_ms[0] / n_prof},
-        }
-        if world == 1 and not args.no_cpu_baseline:
-            tps, ms, desc, cores = _oracle_sample(shape, tmpl, args.cpu_samples, 1, args.planted)
-            line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
-                                    "ms_per_step": ms}
-        print(json.dumps(line))
     ctx.close()
+
+    # ---- the same library in autoregressive mode (no tree, no mask tokens: one row, one token per pass),
+    # the denominator of the paper's speedup metric (Sec. 4.1, "Evaluation Settings")
+    ar = Bita(shape, weights, synth.empty_template(with_group=False), C_max=shape.prompt_len + total_steps + 80,
+              device=dev)
+    start(ar)
+    for s in range(W):
+        ar.step_enqueue(None)
+    barrier()
+    e0.record()
+    for s in range(K):
+        ar.step_enqueue(None)
+    e1.record()
+    barrier()
+    ar_ms = e0.elapsed_time(e1) / K
+    ar.step_finish()
+    ar.close()
+    del ctx, ar, weights, trees_dev
+    torch.cuda.empty_cache()
+    return dict(dev_ms=dev_ms, e2e_ms=e2e_ms, tokens=tokens_timed, emitted=emitted, step_wall=step_wall,
+                launches=launches, fam_ms=fam_ms, fam_n=fam_n, n_prof=n_prof, clocks=clocks, ar_ms=ar_ms, rows=rows)
+
+
+def summarise(shape, tmpl, K, W, fraction, world, m, dev_ms, e2e_ms, total_tokens):
+    """Numbers of one workload as they go into the JSON line."""
+    peak, peak_src = _peaks()
+    weight_bytes = shape.streamed_params * 2
+    fam_ms, fam_n, n_prof, emitted = m["fam_ms"], m["fam_n"], m["n_prof"], m["emitted"]
+    gemm_ms = fam_ms[0] / max(1, fam_n[0])                    # average projection launch
+    gemm_bytes = weight_bytes / (fam_n[0] / n_prof)            # algorithmic bytes of an average launch
+    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
+    mean_C = shape.prompt_len + sum(emitted[:W]) + sum(emitted[W:]) / 2
+    step_bytes = weight_bytes + shape.kv_bytes_per_token() * mean_C
+    step_ms = dev_ms / K
+    value = total_tokens / (dev_ms * 1e-3)
+    ar_tps = world * 1e3 / m["ar_ms"]
+    return {
+        "value": value, "ms_per_step": step_ms, "tokens_per_step": m["tokens"] / K,
+        "tokens_per_step_expected": _expected_tokens_per_step(tmpl, fraction),
+        "step_hbm_frac": (step_bytes / (step_ms * 1e-3) / 1e9) / peak,
+        "step_algorithmic_bytes": step_bytes,
+        "autoregressive": {"ms_per_token": m["ar_ms"], "tokens_per_s": ar_tps, "rows": 1,
+                           "hbm_frac": (weight_bytes + shape.kv_bytes_per_token() * mean_C) / (m["ar_ms"] * 1e-3) / 1e9 / peak},
+        "greedy_speedup": value / ar_tps,
+        "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
+                "p50_ms": statistics.median(m["step_wall"]),
+                "p90_ms": sorted(m["step_wall"])[int(0.9 * (len(m["step_wall"]) - 1))],
+                "h2d_bytes_per_step": 4 * tmpl.N, "d2h_bytes_per_step": 4 * (5 + 2 * 16 + 1 + 160)},
+        "gpu_launches": m["launches"],
+        "clocks": m["clocks"],
+        "roofline": {"bound": "hbm",
+                     "kernel": "k_gemm_tc (weight-streaming projection), mean over the step's launches; CUDA events on "
+                               "the library's stream at the boundaries of runs of consecutive projections",
+                     "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                     "frac": achieved / peak, "algorithmic_bytes_per_launch": gemm_bytes,
+                     "traffic": _traffic_per_mean_launch(shape, tmpl),
+                     "traffic_source": "dram bytes of an earlier ncu capture (profiles/), not measured by this run"
+                                       if _traffic_per_mean_launch(shape, tmpl) else None,
+                     "attention_ms_per_step": fam_ms[1] / n_prof, "projection_ms_per_step": fam_ms[0] / n_prof},
+    }
+
+
+def run_ours(args, names):
+    """`names`: workloads to measure; the LAST one is the headline of the JSON line, the others are
+    reported under `other_workloads`."""
+    from paper_2401_12522_b200.build import build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    K, W = args.steps, args.warmup
+    results = {}
+    for name in names:
+        shape = synth.CONFIGS[name]
+        if args.layers:
+            shape = shape.with_layers(args.layers)
+        tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+        m = measure_workload(shape, tmpl, K, W, args.planted, rank, world, local, dist)
+        dev_ms, e2e_ms, total_tokens = aggregate_over_ranks(dist, world, m["dev_ms"], m["e2e_ms"], m["tokens"], dev)
+        if rank == 0:
+            r = summarise(shape, tmpl, K, W, args.planted, world, m, dev_ms, e2e_ms, total_tokens)
+            r["config"] = _config(shape, tmpl, args.planted, world)
+            if world == 1 and not args.no_cpu_baseline:
+                r["cpu_baseline"] = oracle_leg(shape, tmpl, args.cpu_samples, 1, args.planted, whole_steps=2)
+            results[name] = r
+    if rank == 0:
+        head = results[names[-1]]
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic"}
+        line.update({k: v for k, v in head.items() if k not in ("value", "ms_per_step")})
+        line["other_workloads"] = {n: results[n] for n in names[:-1]}
+        print(json.dumps(line))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -495,16 +616,29 @@ def run_next_rows(args, shape):
         ctx.close()
 
 
+def _spawn_ranks(n: int):
+    """`python bench.py --gpus N` without a launcher: start the N ranks ourselves (one process per GPU)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.exit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="7b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default="all", choices=sorted(synth.CONFIGS) + ["all"],
+                    help="all (default): the 70B shape is the headline, 7B and 13B ride along under other_workloads")
     ap.add_argument("--layers", type=int, default=0, help="truncate the layer stack (debugging only)")
     ap.add_argument("--planted", type=float, default=0.6)
-    ap.add_argument("--cpu-samples", type=int, default=12)
+    ap.add_argument("--cpu-samples", type=int, default=12,
+                    help="cpu_baseline: layer samples of the 70B estimate (whole passes of smaller models: 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--attn-sweep", action="store_true", help="time the tree-attention kernel alone over the sweep shapes")
     ap.add_argument("--next-rows", action="store_true",
@@ -514,19 +648,24 @@ def main():
         run_attn_sweep()
         return
     if args.next_rows:
-        shape = synth.CONFIGS[args.workload]
+        shape = synth.CONFIGS["7b" if args.workload == "all" else args.workload]
         run_next_rows(args, shape.with_layers(args.layers) if args.layers else shape)
         return
     if args.warmup < 3:
         args.warmup = 3
-    shape = synth.CONFIGS[args.workload]
-    if args.layers:
-        shape = shape.with_layers(args.layers)
-    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    world = os.environ.get("WORLD_SIZE")
+    if world is None and args.gpus > 1:
+        _spawn_ranks(args.gpus)
+    if world is not None and int(world) != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started WORLD_SIZE={world} ranks")
+    names = ["7b", "13b", "70b"] if args.workload == "all" else [args.workload]
     if args.impl == "reference":
-        run_reference(args, shape, tmpl)
+        shape = synth.CONFIGS[names[-1]]
+        if args.layers:
+            shape = shape.with_layers(args.layers)
+        run_reference(args, shape, synth.product_rule_template(shape.tree_K, shape.tree_B))
     else:
-        run_ours(args, shape, tmpl)
+        run_ours(args, names)
 
 
 if __name__ == "__main__":

@@ -159,6 +159,32 @@ int bita_rewind(bita_ctx* ctx, bita_kv* kv, int32_t new_len, int32_t last_token)
  * `bytes` must hold L * BITA_MAX_ROWS * d + BITA_MAX_ROWS * V floats. */
 int bita_set_debug_buffer(bita_ctx* ctx, void* dev_buf, size_t bytes);
 
+/* Read back what the most recent pass left for inspection (Algorithm 1 names the quantities: the
+ * output logits L^t, and the top-k predictions of the mask tokens that form C^t), into HOST memory:
+ *   BITA_DEBUG_LOGITS       fp32 [rows][V]     logits of every row of the pass
+ *   BITA_DEBUG_TOPK         int32 [rows][BITA_MAX_TOPK]  selected token ids per row: slot 0 = argmax;
+ *                           slots 1.. are filled for mask rows only, up to the template's k
+ *   BITA_DEBUG_HIDDEN + l   fp32 [rows][d]     residual stream after decoder layer l
+ * rows = rows of that pass.  Logits and hidden states need a debug buffer set BEFORE the pass
+ * (bita_set_debug_buffer: the caller owns all device memory, so it provides the storage).  Waits
+ * for the stream.  `bytes` = capacity of dst; BITA_ERR_INVALID_ARG when too small, when no pass
+ * has run, or when the quantity was not recorded. */
+#define BITA_DEBUG_LOGITS 1
+#define BITA_DEBUG_TOPK 2
+#define BITA_DEBUG_HIDDEN 1000
+int bita_debug_fetch(bita_ctx* ctx, int what, void* dst, size_t bytes);
+
+/* Bound of every device-side wait (mbarriers, split-K counters, cluster hand-overs) of later passes,
+ * in nanoseconds; default 2 s.  A wait that runs out sets the context's status word: the pass
+ * returns BITA_ERR_TIMEOUT, and so does every later one until bita_reset. */
+int bita_set_wait_limit(bita_ctx* ctx, uint64_t limit_ns);
+
+/* Self-check of that mechanism: runs one thread through the library's bounded wait on a barrier
+ * nobody arrives on, with the given limit (1 us .. 1 s).  The wait must give up, so the expected
+ * return value is BITA_ERR_TIMEOUT, and the context's status word is set as after a real timeout
+ * (clear it with bita_reset).  Returns 0 if the wait did not report, which would be a defect. */
+int bita_probe_wait_timeout(bita_ctx* ctx, uint64_t limit_ns);
+
 /* Per-kernel-family device timing of later passes, for roofline reports.  When on, a pass records
  * a CUDA event on the context's stream wherever the kernel family changes, so that every run of
  * consecutive launches of one family (e.g. O, gate/up, down and the next layer's q/k/v projection)
@@ -183,7 +209,7 @@ int bita_last_cuda_error(void);
 /* ---- single operators of the step, exported for per-kernel parity and timing ---- */
 
 /* Y[m][n] = sum_k X[m][k] * W[n][k]  (the small-M weight-streaming projection of the
- * decoder, "memory-bandwidth cost" argument of Sec. 3.2).  X: DEVICE bf16 [M][K],
+ * decoder; Sec. 3.2, last paragraph: the pass is bound by memory traffic, not arithmetic).  X: DEVICE bf16 [M][K],
  * W: DEVICE bf16 [N][K], Y: DEVICE fp32 [M][N].  1 <= M <= BITA_MAX_ROWS, K % 8 == 0.
  * `workspace` DEVICE scratch of bita_gemm_workspace_bytes(M, N, K), 256-byte aligned. */
 int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes);
@@ -199,11 +225,16 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
  *   ctx_len     DEVICE int32 [B]: C per sequence, C + M <= C_max
  *   out    DEVICE bf16 [B][M][H*D]
  * `workspace` DEVICE scratch of bita_attention_workspace_bytes, 256-byte aligned: room for the
- * partial results of the key slices.  (The slices normally run as one thread-block cluster and
- * merge on chip; the scratch is written only when that launch form is refused and a second
- * kernel has to merge.)  A wait between key slices that runs out (2 s) leaves wrong output
- * rather than a hang. */
+ * partial results of the key slices; 0 bytes (workspace may be NULL) when the launch takes a
+ * single key slice.  (The slices normally run as one thread-block cluster and merge on chip; the
+ * scratch is written when that launch form is refused, or when bita_set_attention_route(1) asks
+ * for it, and a second kernel merges.)  A wait between key slices that runs out (2 s) leaves
+ * wrong output rather than a hang. */
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes);
+/* Diagnostic, process-wide: 0 (default) = key slices merge inside a thread-block cluster whenever
+ * that launch form is accepted; 1 = always through the workspace and the separate merge kernel.
+ * Affects bita_tree_attention and the passes of every context. */
+int bita_set_attention_route(int route);
 int bita_tree_attention(const void* q, const void* k, const void* v, const uint32_t* vis,
                         const void* prompt_k, const void* prompt_v, const uint8_t* sees_prompt,
                         const int32_t* ctx_len, void* out, int32_t B, int32_t M, int32_t H,
@@ -224,7 +255,11 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
  * Limits and rules
  *   - The scratch needed is what bita_attention_workspace_bytes reports for (B, M, H, D).  If that
  *     exceeds BITA_STATIC_SCRATCH_BYTES the call returns BITA_ERR_STATIC_SCRATCH and launches
- *     nothing.  (7B-shaped steps, H = 32, M = 69, D = 128, B = 1, fit; large batches do not.)
+ *     nothing.  (7B-shaped steps, H = 32, M = 69, D = 128, B = 1, need 4.6 MB and fit; 133 rows
+ *     at that head count do not.  Launches with so many (sequence, head) pairs that each takes a
+ *     single key slice need no scratch and are always accepted.)
+ *   - With more than one key slice this entry always takes the workspace route: the slices write
+ *     their partial results into the array and a merge kernel reads them back (two launches).
  *   - The first call on each device looks up the array's device address (one runtime query, no
  *     allocation).  Make that first call outside any stream capture.
  *   - The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.

@@ -6,7 +6,7 @@ use of any name below loads the library and raises ImportError if it has not bee
 (``python -m paper_2401_12522_b200.build``).  The ``build`` submodule itself imports without it.
 """
 _NAMES = ("Bita", "BitaError", "StepOut", "lib", "bita_gemm_bf16", "bita_tree_attention",
-          "bita_tree_attention_static", "MAX_ROWS", "MAX_NODES", "MAX_TOPK", "MAX_DEPTH")
+          "bita_tree_attention_static", "set_attention_route", "MAX_ROWS", "MAX_NODES", "MAX_TOPK", "MAX_DEPTH")
 __all__ = list(_NAMES)
 
 

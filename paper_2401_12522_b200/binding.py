@@ -60,6 +60,10 @@ def _signatures():
         "bita_reset": [vp, C.POINTER(KV)],
         "bita_rewind": [vp, C.POINTER(KV), i32, i32],
         "bita_set_debug_buffer": [vp, vp, sz],
+        "bita_debug_fetch": [vp, C.c_int, vp, sz],
+        "bita_set_wait_limit": [vp, C.c_uint64],
+        "bita_probe_wait_timeout": [vp, C.c_uint64],
+        "bita_set_attention_route": [C.c_int],
         "bita_set_kernel_timing": [vp, C.c_int],
         "bita_get_kernel_timing": [vp, C.POINTER(C.c_float), C.POINTER(i32)],
         "bita_block_rows": [vp],
@@ -218,6 +222,27 @@ class Bita:
         off = self.shape.L * MAX_ROWS * self.shape.d
         return self._debug[off: off + rows * self.shape.V].view(rows, self.shape.V)
 
+    DEBUG_LOGITS, DEBUG_TOPK, DEBUG_HIDDEN = 1, 2, 1000
+
+    def debug_fetch(self, what: int, rows: int) -> torch.Tensor:
+        """What the last pass left behind, read back to the host through bita_debug_fetch."""
+        if what == self.DEBUG_TOPK:
+            out = torch.empty((rows, MAX_TOPK), dtype=torch.int32)
+        elif what == self.DEBUG_LOGITS:
+            out = torch.empty((rows, self.shape.V), dtype=torch.float32)
+        else:
+            out = torch.empty((rows, self.shape.d), dtype=torch.float32)
+        _check(lib.bita_debug_fetch(self._ctx, what, C.c_void_p(out.data_ptr()), out.numel() * out.element_size()),
+               "bita_debug_fetch")
+        return out
+
+    def set_wait_limit(self, limit_ns: int):
+        _check(lib.bita_set_wait_limit(self._ctx, int(limit_ns)), "bita_set_wait_limit")
+
+    def probe_wait_timeout(self, limit_ns: int) -> int:
+        """Returns the status the self-check leaves (-6 = the bounded wait gave up, as it must)."""
+        return lib.bita_probe_wait_timeout(self._ctx, int(limit_ns))
+
     def set_kernel_timing(self, on: bool):
         _check(lib.bita_set_kernel_timing(self._ctx, 1 if on else 0), "bita_set_kernel_timing")
 
@@ -265,15 +290,20 @@ def bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, 
     C_max = k.shape[2]
     need = C.c_size_t(0)
     _check(lib.bita_attention_workspace_bytes(B, M, H, D, C.byref(need)), "bita_attention_workspace_bytes")
-    if workspace is None:
+    if workspace is None and need.value:
         workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=q.device)
-    wp = (workspace.data_ptr() + 255) // 256 * 256
+    wp = 0 if workspace is None else (workspace.data_ptr() + 255) // 256 * 256
     if out is None:
         out = torch.empty((B, M, H * D), dtype=torch.bfloat16, device=q.device)
     _check(lib.bita_tree_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(vis), _ptr(prompt_k), _ptr(prompt_v),
                                    _ptr(sees_prompt), _ptr(ctx_len), _ptr(out), B, M, H, H_kv, D, P, C_max,
                                    C.c_void_p(wp), need.value, _stream_handle(stream)), "bita_tree_attention")
     return out
+
+
+def set_attention_route(route: int):
+    """0 = key slices merge inside a thread-block cluster (default), 1 = always through the workspace."""
+    _check(lib.bita_set_attention_route(int(route)), "bita_set_attention_route")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

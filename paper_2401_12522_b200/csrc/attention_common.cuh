@@ -35,6 +35,7 @@ struct AttnArgs {
                              // and merge through distributed shared memory; 0: they leave partial
                              // results in part_ml / part_acc for k_attn_merge
   int32_t* status;           // sticky error word for a wait that ran out (may be null)
+  unsigned long long wait_ns;  // bound of every device-side wait of the launch
 };
 
 // Merge the S slices of each (sequence, head, row) in slice order; write bf16 [B][M][H*D].

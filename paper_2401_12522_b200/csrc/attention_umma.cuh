@@ -78,7 +78,8 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
 }
 // Bounded wait with cluster-scope acquire (the data were written by other CTAs of the cluster).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int32_t* status,
+                                                  unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t i = 0;; ++i) {
     uint32_t ok;
@@ -93,7 +94,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     if ((i & 63u) == 63u) {
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > TC_WAIT_LIMIT_NS) break;
+      else if (now - t0 > limit_ns) break;
     }
   }
   atomicExch(status, BITA_ERR_TIMEOUT);
@@ -182,6 +183,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   }
   const uint32_t tmem = tmem_slot;
   int32_t* status = a.status ? a.status : &status_local;
+  const unsigned long long wait_ns = a.wait_ns;
   if (threadIdx.x == 0) pdl_launch();
 
   // ---- key chunks of this slice (the context length was settled by an earlier pass)
@@ -242,21 +244,21 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     // waits for the S of chunk j-1, then V(j) for the PV of chunk j-2, in that order.
     for (int j = 0; j < n && ok; ++j) {
       if (j + 1 < n && j + 1 >= k_issued) {
-        if (j + 1 >= 2) ok = mbar_wait(smem_u32(&bar_k_empty[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status);
+        if (j + 1 >= 2) ok = mbar_wait(smem_u32(&bar_k_empty[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status, wait_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (lane == 0) issue_tile(j + 1, false);
         k_issued = j + 2;
       }
       if (j >= v_issued) {
-        if (j >= 2) ok = mbar_wait(smem_u32(&bar_v_empty[j & 1]), ((uint32_t)(j >> 1) & 1u) ^ 1u, status);
+        if (j >= 2) ok = mbar_wait(smem_u32(&bar_v_empty[j & 1]), ((uint32_t)(j >> 1) & 1u) ^ 1u, status, wait_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (lane == 0) issue_tile(j, true);
         v_issued = j + 1;
       }
       if (j == fix) {
-        ok = mbar_wait(smem_u32(&bar_v_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
+        ok = mbar_wait(smem_u32(&bar_v_full[j & 1]), (uint32_t)(j >> 1) & 1u, status, wait_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const int live_rows = n_cache - chunk_of(j) * AU_KEYS;
@@ -292,24 +294,24 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
         umma_commit(smem_u32(&bar_s_full[j & 1]));
         if (t == RT - 1) umma_commit(smem_u32(&bar_k_empty[i & 1]));      // the K tile has served every row tile
       };
-      ok = mbar_wait(smem_u32(&bar_q), 0, status);
-      if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, status);
+      ok = mbar_wait(smem_u32(&bar_q), 0, status, wait_ns);
+      if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, status, wait_ns);
       tc_fence_after();
       if (ok) issue_s(0);
       for (int j = 0; j < n_steps && ok; ++j) {
         if (j + 1 < n_steps) {                                            // S of the next step while this one is in softmax
           const int i1 = (j + 1) / RT;
-          if ((j + 1) % RT == 0) ok = mbar_wait(smem_u32(&bar_k_full[i1 & 1]), (uint32_t)(i1 >> 1) & 1u, status);
+          if ((j + 1) % RT == 0) ok = mbar_wait(smem_u32(&bar_k_full[i1 & 1]), (uint32_t)(i1 >> 1) & 1u, status, wait_ns);
           if (ok && j + 1 >= 2)
-            ok = mbar_wait(smem_u32(&bar_s_free[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status);
+            ok = mbar_wait(smem_u32(&bar_s_free[(j + 1) & 1]), ((uint32_t)((j + 1) >> 1) & 1u) ^ 1u, status, wait_ns);
           if (!ok) break;
           tc_fence_after();
           issue_s(j + 1);
         }
         const int i = j / RT, t = j - i * RT;
-        ok = mbar_wait(smem_u32(&bar_p_full), (uint32_t)j & 1u, status);
-        if (ok && t == 0) ok = mbar_wait(smem_u32(&bar_v_full[i & 1]), (uint32_t)(i >> 1) & 1u, status);
-        if (ok && t == 0 && i == fix) ok = mbar_wait(smem_u32(&bar_vfix), 0, status);
+        ok = mbar_wait(smem_u32(&bar_p_full), (uint32_t)j & 1u, status, wait_ns);
+        if (ok && t == 0) ok = mbar_wait(smem_u32(&bar_v_full[i & 1]), (uint32_t)(i >> 1) & 1u, status, wait_ns);
+        if (ok && t == 0 && i == fix) ok = mbar_wait(smem_u32(&bar_vfix), 0, status, wait_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vs = kv_s + (uint32_t)(i & 1) * 2 * TILE + TILE;
@@ -393,7 +395,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
           }
         }
       }
-      if (ok) ok = mbar_wait(smem_u32(&bar_s_full[j & 1]), (uint32_t)(j >> 1) & 1u, status);
+      if (ok) ok = mbar_wait(smem_u32(&bar_s_full[j & 1]), (uint32_t)(j >> 1) & 1u, status, wait_ns);
       ok = __all_sync(0xffffffffu, ok);                         // warp-uniform from here on
       tc_fence_after();
       const uint32_t s_addr = lane_addr + COL_S + (uint32_t)(j & 1) * AU_KEYS + (uint32_t)(g * HK);
@@ -422,7 +424,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       const float sub = m_new == -INFINITY ? 0.f : m_new;
       const float corr = exp2f(m_old - sub);                    // 0 while nothing was seen before
       // P overwrites the tile the previous P V product reads, and the rescale touches an accumulator
-      if (j > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status);
+      if (j > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(j - 1) & 1u, status, wait_ns);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       // P = exp2(s * scale - max), half-row sum, bf16 tile (this thread's 64 keys are one swizzle atom)
@@ -455,7 +457,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       tc_fence_before();
       mbar_arrive_cta(smem_u32(&bar_p_full));
     }
-    if (n_steps > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(n_steps - 1) & 1u, status);
+    if (n_steps > 0 && ok) ok = mbar_wait(smem_u32(&bar_pv_done), (uint32_t)(n_steps - 1) & 1u, status, wait_ns);
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     pdl_wait();
@@ -528,7 +530,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
       asm volatile("fence.acq_rel.cluster;" ::: "memory");
       for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_in), (uint32_t)p));
     }
-    mbar_wait_cluster(smem_u32(&bar_cl_in), 0, status);
+    mbar_wait_cluster(smem_u32(&bar_cl_in), 0, status, wait_ns);
     constexpr int VW = D / 32;
     const int rows_here = min(RT * AU_ROWS, a.M - row0);
     const int r_lo = (int)((long)rows_here * s / a.S), r_hi = (int)((long)rows_here * (s + 1) / a.S);
@@ -588,7 +590,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     if (threadIdx.x == 0) {
       for (int p = 0; p < a.S; ++p) mbar_arrive_remote(mapa_u32(smem_u32(&bar_cl_out), (uint32_t)p));
     }
-    mbar_wait_cluster(smem_u32(&bar_cl_out), 0, status);
+    mbar_wait_cluster(smem_u32(&bar_cl_out), 0, status, wait_ns);
   }
   if (warp == 8) {
     tc_fence_after();

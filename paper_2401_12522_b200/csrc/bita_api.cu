@@ -279,19 +279,39 @@ struct GemmDesc {
 constexpr int GEMM_MAX_CTAS = 296;       // size of the exchange buffer: two CTAs on each of up to 148 SMs
 constexpr int GEMM_MAX_SPLITS = 8;
 
+// What the library remembers per device of the process: CUDA keeps function attributes and
+// device properties per device, so none of this may be a process-wide flag.
+constexpr int MAX_DEVICES = 64;
+struct DeviceFacts {
+  int sms = 0;
+  bool gemm_attr = false, attn_attr = false, select_attr = false;
+  void* static_scratch = nullptr;
+};
+DeviceFacts g_device[MAX_DEVICES];
+DeviceFacts g_device_overflow;          // devices beyond MAX_DEVICES: looked up every time
+
+DeviceFacts* device_facts() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+    g_device_overflow = DeviceFacts();
+    return &g_device_overflow;
+  }
+  return &g_device[dev];
+}
+
 // SMs of the current device (the splits of a launch wait for one another, so a launch with splits
 // never has more CTAs than the GPU holds at once); capped at what the exchange buffer is sized for.
 int sm_count() {
-  static int n = 0;
-  if (!n) {
+  DeviceFacts* f = device_facts();
+  if (!f->sms) {
     int dev = 0, v = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
         cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v > GEMM_MAX_CTAS / 2 ? GEMM_MAX_CTAS / 2 : v;
+      f->sms = v > GEMM_MAX_CTAS / 2 ? GEMM_MAX_CTAS / 2 : v;
     else
-      n = 1;
+      f->sms = 1;
   }
-  return n;
+  return f->sms;
 }
 
 int gemm_splits(int tiles, int K, int max_splits) {
@@ -326,11 +346,12 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
 // Launch: X bf16 (first M rows valid) times the described weights; `p` carries the epilogue.
 int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M, GemmTcParams p, bool pdl,
                    cudaStream_t stream) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  DeviceFacts* facts = device_facts();
+  if (!facts->gemm_attr) {
     CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
-    attr_set = true;
+    facts->gemm_attr = true;
   }
+  if (!p.wait_ns) p.wait_ns = TC_WAIT_LIMIT_NS;
   int splits = g.splits;
   p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.dual = g.dual;
   int cols = 32;
@@ -444,6 +465,8 @@ struct bita_ctx {
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
   std::map<std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>, AttnMaps> attn_map_cache;
   bool pdl;                             // programmatic dependent launch between the kernels of a pass
+  unsigned long long wait_ns;           // bound of every device-side wait
+  int last_rows;                        // rows of the most recent pass (what the debug buffer holds)
 
   // optional per-family event timing
   bool timing;
@@ -486,6 +509,7 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
     it = c->act_maps.emplace(key, m).first;
   }
   p.status = &c->b.state->status;
+  p.wait_ns = c->wait_ns;
   p.part = c->b.gemm_part;
   p.tile_counters = c->b.gemm_cnt;
   mark(c, 0);
@@ -527,7 +551,15 @@ int attn_maps(const AttnArgs& a, std::map<AttnMapKey, AttnMaps>* cache, AttnMaps
 
 // Fills the launch-shape fields of `a` (row_tiles, S, scale) and launches the slices (and the merge
 // kernel where the slices cannot merge themselves).
-int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache) {
+// `route`: ATTN_ROUTE_AUTO merges the slices inside a thread-block cluster and falls back to the
+// workspace route only when that launch form is refused; ATTN_ROUTE_WORKSPACE always sends the
+// partial results through a.part_ml / a.part_acc and the merge kernel.
+enum { ATTN_ROUTE_AUTO = 0, ATTN_ROUTE_WORKSPACE = 1 };
+int g_attention_route = ATTN_ROUTE_AUTO;      // process-wide diagnostic switch (bita_set_attention_route)
+
+int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache,
+                     int route = -1) {
+  if (route < 0) route = g_attention_route;
   attn_shape(a.H, a.B, a.M, &a.row_tiles, &a.S);
   AttnMaps maps;
   {
@@ -538,13 +570,14 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
   const int RT = a.M > AU_ROWS ? 2 : 1;                          // row tiles per CTA
   const size_t tile = (size_t)(a.D / 64) * AU_ATOM;
   const size_t smem = (RT + 4) * tile + 2 * AU_ATOM + 1024;       // Q (RT tiles), 2 x (K, V), P
-  static bool attr_set = false;
-  if (!attr_set) {
+  DeviceFacts* facts = device_facts();
+  if (!a.wait_ns) a.wait_ns = TC_WAIT_LIMIT_NS;
+  if (!facts->attn_attr) {
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-    attr_set = true;
+    facts->attn_attr = true;
   }
   dim3 g1(a.H, a.S, a.B * a.row_tiles), g2(a.M, a.H, a.B);
   auto run = [&](unsigned cluster_y) {
@@ -556,12 +589,15 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
   };
   if (n_launched) *n_launched = 1;
   if (a.S == 1) return run(1);
-  a.cluster = 1;
-  int rc = run((unsigned)a.S);
-  if (rc == BITA_OK) return rc;
-  // The cluster launch was refused: the slices leave their partial results in global memory
-  // and a second kernel merges them.
-  (void)cudaGetLastError();
+  int rc;
+  if (route != ATTN_ROUTE_WORKSPACE) {
+    a.cluster = 1;
+    rc = run((unsigned)a.S);
+    if (rc == BITA_OK) return rc;
+    // The cluster launch was refused: the slices leave their partial results in global memory
+    // and a second kernel merges them.
+    (void)cudaGetLastError();
+  }
   a.cluster = 0;
   if (n_launched) *n_launched = 2;
   if ((rc = run(1))) return rc;
@@ -578,6 +614,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   Buffers& b = c->b;
   c->ev_family.clear();
   c->ev_count.clear();
+  c->last_rows = M;
   mark(c, 2);
   const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
   const bool pdl = c->pdl;
@@ -631,6 +668,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
     a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
     a.status = &b.state->status;
+    a.wait_ns = c->wait_ns;
     {
       mark(c, 1);
       int n = 0;
@@ -649,10 +687,10 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     {
       const size_t row_bytes = (size_t)m.V * 4;
       const int use_smem = row_bytes <= 200 * 1024 ? 1 : 0;
-      static bool sel_attr = false;
-      if (!sel_attr) {
+      DeviceFacts* facts = device_facts();
+      if (!facts->select_attr) {
         CU_TRY(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        sel_attr = true;
+        facts->select_attr = true;
       }
       mark(c, 2);
       if ((rc = launch(s, pdl, dim3(M), dim3(1024), use_smem ? row_bytes : 0, 1, k_select, P, (const float*)b.logits,
@@ -733,6 +771,8 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   c->launches = 0;
   c->timing = false;
   c->pdl = getenv("BITA_NO_PDL") == nullptr;
+  c->wait_ns = TC_WAIT_LIMIT_NS;
+  c->last_rows = 0;
 
   c->prefilled = false;
   c->len_upper = 0;
@@ -777,6 +817,8 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
 
 int bita_reset(bita_ctx* c, bita_kv* kv) {
   if (!c || !kv) return BITA_ERR_INVALID_ARG;
+  // a pass that gave up on a wait may have left split counters half way
+  CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream));
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   CU_TRY(cudaStreamSynchronize(c->stream));
   c->prefilled = false;
@@ -881,6 +923,47 @@ int bita_set_debug_buffer(bita_ctx* c, void* dev_buf, size_t bytes) {
   return BITA_OK;
 }
 
+int bita_debug_fetch(bita_ctx* c, int what, void* dst, size_t bytes) {
+  if (!c || !dst) return BITA_ERR_INVALID_ARG;
+  const size_t rows = (size_t)c->last_rows;
+  const void* src = nullptr;
+  size_t need = 0;
+  if (what == BITA_DEBUG_TOPK) {
+    src = c->b.sel_id;
+    need = rows * BITA_MAX_TOPK * 4;
+  } else if (what == BITA_DEBUG_LOGITS) {
+    if (!c->dbg) return BITA_ERR_INVALID_ARG;
+    src = c->dbg + (size_t)c->m.L * BITA_MAX_ROWS * c->m.d;
+    need = rows * c->m.V * 4;
+  } else if (what >= BITA_DEBUG_HIDDEN && what < BITA_DEBUG_HIDDEN + c->m.L) {
+    if (!c->dbg) return BITA_ERR_INVALID_ARG;
+    src = c->dbg + (size_t)(what - BITA_DEBUG_HIDDEN) * BITA_MAX_ROWS * c->m.d;
+    need = rows * c->m.d * 4;
+  } else {
+    return BITA_ERR_INVALID_ARG;
+  }
+  if (rows == 0 || bytes < need) return BITA_ERR_INVALID_ARG;
+  CU_TRY(cudaMemcpyAsync(dst, src, need, cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  return BITA_OK;
+}
+
+int bita_set_wait_limit(bita_ctx* c, uint64_t limit_ns) {
+  if (!c || limit_ns < 1000 || limit_ns > 10000000000ull) return BITA_ERR_INVALID_ARG;
+  c->wait_ns = limit_ns;
+  return BITA_OK;
+}
+
+int bita_probe_wait_timeout(bita_ctx* c, uint64_t limit_ns) {
+  if (!c || limit_ns < 1000 || limit_ns > 1000000000ull) return BITA_ERR_INVALID_ARG;
+  k_wait_probe<<<1, 32, 0, c->stream>>>(&c->b.state->status, (unsigned long long)limit_ns);
+  CU_TRY(cudaGetLastError());
+  int32_t status = 0;
+  CU_TRY(cudaMemcpyAsync(&status, &c->b.state->status, 4, cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(cudaStreamSynchronize(c->stream));
+  return status;
+}
+
 int bita_set_kernel_timing(bita_ctx* c, int on) {
   if (!c) return BITA_ERR_INVALID_ARG;
   c->timing = on != 0;
@@ -967,32 +1050,49 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
   if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
   const size_t S = attn_splits(H, B, M);
-  *out_bytes = align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
+  // a single key slice writes its output itself and needs no scratch at all
+  *out_bytes = S == 1 ? 0 : align_up((size_t)B * H * S * M * 2 * 4) + align_up((size_t)B * H * S * M * D * 4);
   return BITA_OK;
 }
 
-int bita_tree_attention(const void* q, const void* k, const void* v, const uint32_t* vis, const void* prompt_k,
+namespace {
+int tree_attention_impl(const void* q, const void* k, const void* v, const uint32_t* vis, const void* prompt_k,
                         const void* prompt_v, const uint8_t* sees_prompt, const int32_t* ctx_len, void* out, int32_t B,
                         int32_t M, int32_t H, int32_t H_kv, int32_t D, int32_t P, int32_t C_max, void* workspace,
-                        size_t workspace_bytes, void* cuda_stream) {
+                        size_t workspace_bytes, void* cuda_stream, int route) {
   size_t need = 0;
   int rc = bita_attention_workspace_bytes(B, M, H, D, &need);
   if (rc) return rc;
   if (!q || !k || !v || !vis || !ctx_len || !out || H_kv < 1 || H % H_kv || P < 0 || P > 64 || C_max < M)
     return BITA_ERR_INVALID_ARG;
   if (P > 0 && (!prompt_k || !prompt_v || !sees_prompt)) return BITA_ERR_INVALID_ARG;
-  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace % ALIGN)) return BITA_ERR_WORKSPACE;
+  if (need > 0 && (!workspace || workspace_bytes < need || ((uintptr_t)workspace % ALIGN))) return BITA_ERR_WORKSPACE;
   AttnArgs a{};
   const int W = (M + 31) / 32;
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
   a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
-  // workspace: partial results of the key slices (used when the slices cannot run as a cluster)
+  // workspace: partial results of the key slices (used when the slices do not merge inside a cluster)
   a.part_ml = (float*)workspace;
   a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr))) return rc;
+  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr, route))) return rc;
   CU_TRY(cudaGetLastError());
+  return BITA_OK;
+}
+}  // namespace
+
+int bita_tree_attention(const void* q, const void* k, const void* v, const uint32_t* vis, const void* prompt_k,
+                        const void* prompt_v, const uint8_t* sees_prompt, const int32_t* ctx_len, void* out, int32_t B,
+                        int32_t M, int32_t H, int32_t H_kv, int32_t D, int32_t P, int32_t C_max, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+  return tree_attention_impl(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
+                             workspace, workspace_bytes, cuda_stream, -1);
+}
+
+int bita_set_attention_route(int route) {
+  if (route != ATTN_ROUTE_AUTO && route != ATTN_ROUTE_WORKSPACE) return BITA_ERR_INVALID_ARG;
+  g_attention_route = route;
   return BITA_OK;
 }
 
@@ -1004,21 +1104,16 @@ int bita_tree_attention(const void* q, const void* k, const void* v, const uint3
 static __device__ __align__(256) unsigned char g_static_scratch[BITA_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int MAX_DEVICES = 64;
-void* g_static_scratch_addr[MAX_DEVICES] = {nullptr};
-
 // Device address of the scratch array on the current device (looked up on first use).
 int static_scratch_address(void** out) {
-  int dev = -1;
-  CU_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= MAX_DEVICES) return BITA_ERR_INVALID_ARG;
-  if (!g_static_scratch_addr[dev]) {
+  DeviceFacts* f = device_facts();
+  if (!f->static_scratch) {
     void* p = nullptr;
     CU_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
     if (!p || ((uintptr_t)p % ALIGN)) return BITA_ERR_CUDA;
-    g_static_scratch_addr[dev] = p;
+    f->static_scratch = p;
   }
-  *out = g_static_scratch_addr[dev];
+  *out = f->static_scratch;
   return BITA_OK;
 }
 }  // namespace
@@ -1032,12 +1127,15 @@ int bita_tree_attention_static(const void* q, const void* k, const void* v, cons
   if (rc) return rc;
   if (need > BITA_STATIC_SCRATCH_BYTES) return BITA_ERR_STATIC_SCRATCH;
   void* scratch = nullptr;
-  rc = static_scratch_address(&scratch);
-  if (rc) return rc;
-  // Every partial result that the merge reads was written by the slices of the same call, so
-  // nothing in the shared array has to be cleared first.
-  return bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
-                             scratch, need, cuda_stream);
+  if (need > 0) {
+    rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+  }
+  // The key slices always leave their partial results in the built-in array and the merge kernel
+  // reads them back (the workspace route).  Every slot the merge reads was written by the slices
+  // of the same call, so nothing in the shared array has to be cleared first.
+  return tree_attention_impl(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, out, B, M, H, H_kv, D, P, C_max,
+                             scratch, need, cuda_stream, ATTN_ROUTE_WORKSPACE);
 }
 
 }  // extern "C"

@@ -12,9 +12,9 @@
 namespace bita {
 
 // ---------------------------------------------------------------------------------------------
-// Packing (Sec. 3.2 "flatten the draft candidate token tree, along with the attached mask
-// tokens"; Appendix B): row 0 = last accepted token, rows 1..N = tree tokens (token -1 -> zero
-// row), then the mask embeddings.  Position ids: C + rel_pos.
+// Packing (Sec. 3.2, Appendix B: the candidate tree and its mask groups become one row sequence):
+// row 0 = last accepted token, rows 1..N = tree tokens (token -1 -> zero row), then the mask
+// embeddings.  Position ids: C + rel_pos.
 // x: fp32 [M][d] residual stream; pos: int32 [M].
 __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int32_t* __restrict__ tree_tokens,
                         const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
@@ -148,8 +148,8 @@ __global__ void __launch_bounds__(1024) k_select(DevPlan plan, const float* __re
 
 // ---------------------------------------------------------------------------------------------
 // Greedy verification (Algorithm 1, else-branch, general-tree form) and next-tree construction
-// (Algorithm 1, "Get C^t by selecting the top k predictions ... of the mask token group linked to
-// the last accepted candidate token").  One warp: lanes scan the children of the current node.
+// (Algorithm 1, last step of the else-branch: the next candidates are the top-k picks of the mask
+// group that hangs on the last accepted node).  One warp: lanes scan the children of the current node.
 __global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t* __restrict__ row_token,
                          const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec) {
   pdl_launch();
@@ -245,8 +245,8 @@ __global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __r
 }
 
 // ---------------------------------------------------------------------------------------------
-// Cache compaction ("its prediction, along with its subsequent tokens, is discarded", Fig. 3
-// caption): the j-th accepted node's entry moves from slot C+1+idx_j to slot C+1+j.  One thread
+// Cache compaction (Fig. 3 caption: rejected drafts and what follows them leave no trace): the
+// j-th accepted node's entry moves from slot C+1+idx_j to slot C+1+j.  One thread
 // owns a 16-byte column chunk and walks j upwards, which is alias-safe because idx_j >= j and
 // idx is increasing along a path.  grid = (L * H_kv), cache layout [L][H_kv][C_max][D].
 __global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, bf16* __restrict__ kc,
@@ -270,6 +270,18 @@ __global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, b
       }
     }
   }
+}
+
+// Diagnostic: one thread runs the library's bounded mbarrier wait on a barrier that nobody ever
+// arrives on, so the wait must run out after `limit_ns`, raise the status word and return.
+__global__ void k_wait_probe(int32_t* __restrict__ status, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, status, limit_ns);
 }
 
 __global__ void k_set_state(DevState* st, int len, int root) {
