@@ -271,6 +271,7 @@ int make_map3(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64
 // One weight matrix (or a gate/up pair) as the projection kernel sees it.
 struct GemmDesc {
   CUtensorMap a0, a1;
+  const void *w0 = nullptr, *w1 = nullptr;
   int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
 };
 
@@ -327,6 +328,8 @@ int gemm_splits(int tiles, int K, int max_splits) {
 int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, int max_splits) {
   g->K = K;
   g->dual = W1 ? 1 : 0;
+  g->w0 = W0;
+  g->w1 = W1;
   int rc;
   if (W1) {           // N = rows of each of the two matrices
     g->tiles = (N + 63) / 64;
@@ -343,6 +346,15 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
   return BITA_OK;
 }
 
+// Split-K factor a launch of `g` takes for a block of n_pad padded rows: blocks past 128 padded
+// rows run one CTA per SM, and then a split only pays while all its CTAs fit in one wave.
+int effective_splits(const GemmDesc& g, int n_pad) {
+  const int sms = sm_count();
+  int splits = g.splits;
+  if (n_pad > 128 && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
+  return splits;
+}
+
 // Launch: X bf16 (first M rows valid) times the described weights; `p` carries the epilogue.
 int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M, GemmTcParams p, bool pdl,
                    cudaStream_t stream) {
@@ -352,7 +364,7 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
     facts->gemm_attr = true;
   }
   if (!p.wait_ns) p.wait_ns = TC_WAIT_LIMIT_NS;
-  int splits = g.splits;
+  int splits = effective_splits(g, n_pad);
   p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.dual = g.dual;
   int cols = 32;
   while (cols < n_pad) cols <<= 1;
@@ -362,16 +374,16 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   // up to 96 rows, 3 beyond); larger ones one per SM, and then a split only pays while all its CTAs
   // fit in one wave.
   const int sms = sm_count();
-  if (n_pad > 128 && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
   const bool two_per_sm = n_pad <= 128 && g.tiles * splits > sms;
   const size_t budget = (two_per_sm ? 110 : 220) * 1024;
-  int stages = (int)((budget - 1024) / stage);
+  const size_t extra = 1024;                                 // alignment slack
+  int stages = (int)((budget - extra) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
   if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // staging of a whole tile
   p.splits = splits;
   p.stages = stages;
-  const size_t smem = stages * stage + 1024;
+  const size_t smem = stages * stage + extra;
   return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc, g.a0, g.a1, map_b, p);
 }
 
@@ -401,7 +413,7 @@ int attn_splits(int H, int B, int M) {
 
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
-  float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; float* logits; unsigned long long* sumsq;
+  float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; unsigned long long* cand; unsigned long long* sumsq;
   int32_t* sel_id; float* sel_val; int32_t* pos; int32_t* row_token; float* part_ml; float* part_acc; float* gemm_part; int32_t* gemm_cnt;
   float2* rope_tab; float2* rope_blk; DevState* state; DevRecord* rec; void* plan_step; void* plan_prefill;
   int32_t* query_tokens; int32_t* tree_in;
@@ -423,7 +435,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.att = (bf16*)take(R * m.H * m.D * 2);
   t.sumsq = (unsigned long long*)take((size_t)(2 * m.L + 1) * R * 8);
   t.hf = (bf16*)take(R * (size_t)m.F * 2);
-  t.logits = (float*)take(R * (size_t)m.V * 4);
+  t.cand = (unsigned long long*)take(R * (size_t)((m.V + TC_BLOCK_N - 1) / TC_BLOCK_N) * BITA_MAX_TOPK * 8);
   t.sel_id = (int32_t*)take(R * BITA_MAX_TOPK * 4);
   t.sel_val = (float*)take(R * BITA_MAX_TOPK * 4);
   t.pos = (int32_t*)take(R * 4);
@@ -573,8 +585,8 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
   DeviceFacts* facts = device_facts();
   if (!a.wait_ns) a.wait_ns = TC_WAIT_LIMIT_NS;
   if (!facts->attn_attr) {
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     CU_TRY(cudaFuncSetAttribute(k_attn_umma<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
     facts->attn_attr = true;
@@ -683,24 +695,21 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
                              cudaMemcpyDeviceToDevice, s));
   }
   if (want_logits) {
-    if ((rc = gemm(c, c->d_head, b.xn, M, with_norm(epi_store(b.logits, m.V), 2 * m.L)))) return rc;
-    {
-      const size_t row_bytes = (size_t)m.V * 4;
-      const int use_smem = row_bytes <= 200 * 1024 ? 1 : 0;
-      DeviceFacts* facts = device_facts();
-      if (!facts->select_attr) {
-        CU_TRY(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        facts->select_attr = true;
-      }
-      mark(c, 2);
-      if ((rc = launch(s, pdl, dim3(M), dim3(1024), use_smem ? row_bytes : 0, 1, k_select, P, (const float*)b.logits,
-                       m.V, use_smem, b.sel_id, b.sel_val)))
-        return rc;
-    }
+    // LM head with the first half of the selection in its epilogue; the logits themselves are kept
+    // only when a debug buffer asks for them.
+    GemmTcParams hp{};
+    hp.mode = EPI_HEAD;
+    hp.out = c->dbg ? c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d : nullptr;
+    hp.ldo = m.V;
+    hp.cand = b.cand;
+    hp.row_kind = P.row_kind;
+    hp.k_max = P.k_max;
+    if ((rc = gemm(c, c->d_head, b.xn, M, with_norm(hp, 2 * m.L)))) return rc;
+    mark(c, 2);
+    if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select_merge, P, (const unsigned long long*)b.cand,
+                     c->d_head.tiles, b.sel_id, b.sel_val)))
+      return rc;
     c->launches += 1;
-    if (c->dbg)
-      CU_TRY(cudaMemcpyAsync(c->dbg + (size_t)m.L * BITA_MAX_ROWS * m.d, b.logits, (size_t)M * m.V * 4,
-                             cudaMemcpyDeviceToDevice, s));
   }
   mark(c, -1);
   CU_TRY(cudaGetLastError());

@@ -45,7 +45,25 @@ enum GemmEpilogue : int32_t {
   EPI_SWIGLU = 1,   // dual tile: hf[m][f] = silu(gate) * up            (bf16)
   EPI_QKV = 2,      // rotary embedding, q -> bf16 buffer, k/v -> cache (bf16)
   EPI_RESID = 3,    // x[m][n] += y; xhat = bf16(x * gain); row sums of x^2 for the next RMSNorm
+  EPI_HEAD = 4,     // LM head: per row, the tile's best entries as ordered keys (and the fp32 logits when asked for)
 };
+
+// Selection key of a logit: larger key = earlier in the order (value descending, token id ascending).
+// The value's bits are mapped so that unsigned comparison follows the float order; a NaN never wins.
+__device__ __forceinline__ unsigned long long select_key(float v, int id) {
+  uint32_t b = __float_as_uint(v);
+  b = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  if (!(v == v)) b = 0u;
+  return ((unsigned long long)b << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)id);
+}
+__device__ __forceinline__ float select_key_value(unsigned long long key) {
+  uint32_t b = (uint32_t)(key >> 32);
+  b = (b & 0x80000000u) ? (b & 0x7FFFFFFFu) : ~b;
+  return __uint_as_float(b);
+}
+__device__ __forceinline__ int select_key_id(unsigned long long key) {
+  return (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
+}
 
 // RMSNorm is split between producer and consumer so that it needs no pass of its own: the
 // projection that updates the residual stream x also writes xhat = bf16(x * gain) and adds its
@@ -80,9 +98,13 @@ struct GemmTcParams {
   const unsigned long long* in_sumsq;
   int32_t norm_d;
   float norm_eps;
-  // EPI_STORE
+  // EPI_STORE, EPI_HEAD (null in EPI_HEAD: the logits are not kept)
   float* out;            // fp32 [M][ldo]
   int32_t ldo;
+  // EPI_HEAD: cand[row][tile][BITA_MAX_TOPK] = the best sel_k(row) keys of the tile's 128 logits, best first
+  unsigned long long* cand;
+  const int32_t* row_kind;   // [M] RowKind: mask rows keep k_max entries, all others one (their argmax)
+  int32_t k_max;
   // EPI_SWIGLU
   bf16* hf;              // bf16 [M][F]
   int32_t F;
@@ -570,7 +592,32 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
           for (int u = 0; u < RB; ++u)
             if (live[u]) atomicAdd(p.out_sumsq + t0 + tb + NW * u, sumsq_to_fixed(ss[u]));
         }
-      } else if (p.mode == EPI_STORE) {
+      } else if (p.mode == EPI_STORE || p.mode == EPI_HEAD) {
+        if (p.mode == EPI_HEAD) {
+          // Per row: the best entries of this tile, picked one at a time by a warp-wide maximum over
+          // ordered keys (a key is unique, so "remove the winner" is an equality test).
+#pragma unroll
+          for (int u = 0; u < RB; ++u) {
+            if (!live[u]) continue;                              // warp-uniform
+            const int row = t0 + tb + NW * u;
+            const int kk = p.row_kind[row] == ROW_MASK ? p.k_max : 1;
+            unsigned long long key[4];
+            const float vals[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) key[e] = n4 + e < p.N ? select_key(vals[e], n4 + e) : 0ull;
+            unsigned long long* dst = p.cand + ((size_t)row * gridDim.x + tile) * BITA_MAX_TOPK;
+            for (int t = 0; t < kk; ++t) {
+              unsigned long long best = max(max(key[0], key[1]), max(key[2], key[3]));
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (key[e] == best) key[e] = 0ull;
+              if (lane == 0) dst[t] = best;
+            }
+          }
+          if (!p.out) continue;
+        }
 #pragma unroll
         for (int u = 0; u < RB; ++u) {
           if (!live[u]) continue;

@@ -66,83 +66,43 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
 }
 
 // ---------------------------------------------------------------------------------------------
-// Argmax / sorted top-k of each logits row, order = (value descending, token id ascending).
-// One block per row; pass t picks the best entry strictly after the previous pick.
-// sel_id: int32 [M][BITA_MAX_TOPK], sel_val: fp32 [M][BITA_MAX_TOPK].
-__device__ __forceinline__ bool before(float v1, int i1, float v2, int i2) {
-  return v1 > v2 || (v1 == v2 && i1 < i2);
-}
-
-__global__ void __launch_bounds__(1024) k_select(DevPlan plan, const float* __restrict__ logits, int V, int use_smem,
-                                                 int32_t* __restrict__ sel_id, float* __restrict__ sel_val) {
+// Second half of the selection that starts in the LM head's epilogue (Algorithm 1: the argmax `a`
+// of a token row, the top k predictions of a mask row): every tile of 128 vocabulary entries has
+// left its best entries of each row as ordered keys; one block per row picks the overall best
+// k of them, again one at a time ("the largest key below the previous pick").
+// cand: [M][tiles][BITA_MAX_TOPK]; sel_id / sel_val as k_select writes them.
+__global__ void __launch_bounds__(256) k_select_merge(DevPlan plan, const unsigned long long* __restrict__ cand, int tiles,
+                                                      int32_t* __restrict__ sel_id, float* __restrict__ sel_val) {
   pdl_launch();
   pdl_wait();
-  extern __shared__ float srow[];            // the row, kept on chip for the later passes (when it fits)
-  __shared__ float sv[32];
-  __shared__ int si[32];
-  __shared__ float pv;
-  __shared__ int pi;
+  __shared__ unsigned long long red[8];
+  __shared__ unsigned long long pick;
   const int r = blockIdx.x;
-  const int kind = plan.row_kind[r];
-  const int K = (kind == ROW_MASK) ? plan.k_max : 1;
-  const float* row = logits + (size_t)r * V;
-  float prev_v = 0.f;
-  int prev_i = -1;
+  const int K = plan.row_kind[r] == ROW_MASK ? plan.k_max : 1;
+  const unsigned long long* row = cand + (size_t)r * tiles * BITA_MAX_TOPK;
+  const int n = tiles * K;                           // entry e: tile e / K, slot e % K
+  unsigned long long prev = ~0ull;
   for (int t = 0; t < K; ++t) {
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    if (t == 0 && (V & 3) == 0) {
-      // first pass: 16-byte loads from global memory, copy to shared memory on the way
-      const float4* row4 = reinterpret_cast<const float4*>(row);
-      for (int c4 = threadIdx.x; c4 < (V >> 2); c4 += blockDim.x) {
-        const float4 q = row4[c4];
-        if (use_smem && K > 1) reinterpret_cast<float4*>(srow)[c4] = q;
-        const float vals[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float v = vals[e];
-          const int c = 4 * c4 + e;
-          if (v == v && before(v, c, bv, bi)) { bv = v; bi = c; }
-        }
-      }
-    } else {
-      const float* src = (t > 0 && use_smem && (V & 3) == 0) ? srow : row;
-      for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        const float v = src[c];
-        if (!(v == v)) continue;
-        if (prev_i >= 0 && !before(prev_v, prev_i, v, c)) continue;  // not strictly after the previous pick
-        if (before(v, c, bv, bi)) { bv = v; bi = c; }
-      }
+    unsigned long long best = 0ull;
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+      const unsigned long long k = row[(size_t)(e / K) * BITA_MAX_TOPK + (e % K)];
+      if (k < prev && k > best) best = k;
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
     __syncthreads();
-    if (threadIdx.x < 32) {
-      const int nw = blockDim.x >> 5;
-      bv = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
-      bi = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-      }
-      if (threadIdx.x == 0) {
-        pv = bv;
-        pi = (bi == 0x7fffffff) ? -1 : bi;
-        sel_id[(size_t)r * BITA_MAX_TOPK + t] = pi;
-        sel_val[(size_t)r * BITA_MAX_TOPK + t] = bv;
-      }
+    if (threadIdx.x == 0) {
+      unsigned long long b = 0ull;
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) b = max(b, red[w]);
+      pick = b;
+      const bool none = (b >> 32) == 0ull;            // nothing left (or only NaN entries)
+      sel_id[(size_t)r * BITA_MAX_TOPK + t] = none ? -1 : select_key_id(b);
+      sel_val[(size_t)r * BITA_MAX_TOPK + t] = none ? -INFINITY : select_key_value(b);
     }
     __syncthreads();
-    prev_v = pv;
-    prev_i = pi;
-    if (prev_i < 0) break;
+    prev = pick;
+    if ((prev >> 32) == 0ull) break;
   }
 }
 
