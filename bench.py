@@ -559,11 +559,32 @@ def run_attn_sweep():
                 del q, k, v, flush
 
 
+def _time_steps(ctx, steps, warm=4):
+    for _ in range(warm):
+        ctx.step_enqueue(None)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        ctx.step_enqueue(None)
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.step_finish()
+    return e0.elapsed_time(e1) / steps
+
+
 def run_next_rows(args, shape):
-    """Measurements beyond the headline step: the first pass (Algorithm 1, t = 1) as a timed path, and
-    the cost side of the template comparison (Sec. 4.3): step latency per tree template at this
-    model shape.  One JSON line each; device-resident, CUDA events, no planted acceptance."""
-    from paper_2401_12522_b200 import Bita
+    """Measurements beyond the headline step, one JSON line each (device-resident, CUDA events):
+
+    * the first pass (Algorithm 1, t = 1) as a timed path;
+    * the cost side of the paper's comparison of decoding methods (Sec. 4.3, Table 4): step latency
+      of every tree template at this model shape - straightforward decoding, fully tree-based
+      decoding with k = 1..4 candidates per mask, the efficient (comb) tree, each with a mask group
+      per node as the paper attaches them, plus the configuration's product-rule tree - next to
+      the library in autoregressive mode.  The acceptance side comes from the stated synthetic model
+      in synth/acceptance.py (no tuned model or dataset exists here): tokens per pass by seeded
+      simulation, tokens/s = tokens per pass / measured latency, speedup = tokens/s over AR tokens/s.
+    """
+    from paper_2401_12522_b200 import Bita, BitaError
     from paper_2401_12522_b200.build import build
     build()
     dev = torch.device("cuda:0")
@@ -571,49 +592,64 @@ def run_next_rows(args, shape):
     peak, _ = _peaks()
     weights = synth.make_weights(shape, MODEL_SEED, dtype=torch.bfloat16, device=dev)
     prompt = synth.uniform_ints(replica_plan(0, shape)["prompt_seed"], 5001, shape.prompt_len, shape.V).tolist()
-    n, steps = shape.n_mask, 24
-    templates = [
-        ("straightforward (chain of top-1 drafts, one group)", synth.chain_template(n)),
-        ("product-rule tree of the configuration, one group", synth.product_rule_template(shape.tree_K, shape.tree_B)),
-        ("efficient comb tree k=5, a group per node (paper default)", synth.comb_template(n, 5)),
-        ("efficient comb tree k=3, a group per node", synth.comb_template(n, 3)),
-    ]
-    for name, tmpl in templates:
-        rows = 1 + tmpl.N + tmpl.G * n
-        depth = max(tmpl.depths(), default=0)
-        C_max = shape.prompt_len + (steps + 8) * (depth + 1) + rows + 64
-        ctx = Bita(shape, weights, tmpl, C_max=C_max, device=dev)
+    steps = 24
+    model = synth.AcceptanceModel()
+    # ---- autoregressive mode: one row, one token per pass
+    ar = Bita(shape, weights, synth.empty_template(with_group=False), C_max=shape.prompt_len + steps + 80, device=dev)
+    ar.prefill(prompt)
+    ar_ms = _time_steps(ar, steps)
+    ar.close()
+    print(json.dumps({"metric": "step_latency_by_template", "workload": shape.name, "template": "autoregressive (no tree, no masks)",
+                      "n_mask": 0, "nodes": 0, "groups": 0, "rows": 1, "ms_per_step": ar_ms, "tokens_per_pass_model": 1.0,
+                      "tokens_per_s": 1e3 / ar_ms, "speedup_vs_autoregressive": 1.0}))
+    # ---- first pass
+    ctx = Bita(shape, weights, synth.product_rule_template(shape.tree_K, shape.tree_B),
+               C_max=shape.prompt_len + 400, device=dev)
+    times = []
+    for it in range(3):
         ctx.reset()
-        # ---- first pass: equal blocks of up to 248 rows through the same kernels, then the first tree
-        times = []
-        for it in range(3):
-            ctx.reset()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            ctx.prefill(prompt)
-            e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        pre_ms = min(times)
-        flops = 2.0 * shape.streamed_params * shape.prompt_len
-        # ---- steps with the model's own drafts (random-init masks: acceptance ~ 0, so this is cost only)
-        for s in range(4):
-            ctx.step_enqueue(None)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for s in range(steps):
-            ctx.step_enqueue(None)
+        ctx.prefill(prompt)
         e1.record()
         torch.cuda.synchronize()
-        ctx.step_finish()
-        ms = e0.elapsed_time(e1) / steps
-        print(json.dumps({"metric": "step_latency_by_template", "workload": shape.name, "template": name,
-                          "nodes": tmpl.N, "groups": tmpl.G, "rows": rows, "ms_per_step": ms,
-                          "weights_gb_per_s": shape.streamed_params * 2 / ms / 1e6,
-                          "hbm_frac": shape.streamed_params * 2 / ms / 1e6 / peak,
-                          "prefill": {"tokens": shape.prompt_len, "ms": pre_ms, "tokens_per_s": shape.prompt_len / pre_ms * 1e3,
-                                      "tflops": flops / pre_ms / 1e9}}))
+        times.append(e0.elapsed_time(e1))
+    ctx.close()
+    pre_ms = min(times)
+    flops = 2.0 * shape.streamed_params * shape.prompt_len
+    print(json.dumps({"metric": "first_pass", "workload": shape.name, "tokens": shape.prompt_len, "ms": pre_ms,
+                      "tokens_per_s": shape.prompt_len / pre_ms * 1e3, "tflops": flops / pre_ms / 1e9}))
+    # ---- templates; n = 3 is the paper's setting for 7B-class models (Sec. 4.1), n = 4 this configuration's
+    cases = []
+    for n in sorted({3, shape.n_mask}):
+        cases += [(n, "straightforward decoding (chain of top-1 drafts, one group after the last token)", synth.chain_template(n))]
+        cases += [(n, f"fully tree-based decoding k={k}, a group per node", synth.full_tree_template(n, k)) for k in (1, 2, 3, 4)]
+        cases += [(n, "efficient tree-based decoding (comb tree k=5, a group per node: the paper's default)",
+                   synth.comb_template(n, 5))]
+    cases += [(shape.n_mask, "product-rule tree of the measured configuration (64 nodes, one group)",
+               synth.product_rule_template(shape.tree_K, shape.tree_B))]
+    for n, name, tmpl in cases:
+        from dataclasses import replace
+        sh = replace(shape, n_mask=n)
+        rows = 1 + tmpl.N + tmpl.G * n
+        acc = synth.tokens_per_pass(tmpl, n, model)["tokens_per_pass"]
+        line = {"metric": "step_latency_by_template", "workload": shape.name, "template": name, "n_mask": n,
+                "nodes": tmpl.N, "groups": tmpl.G, "rows": rows, "tokens_per_pass_model": acc,
+                "acceptance_model": {"h0": model.h0, "gamma": model.gamma, "r": model.r}}
+        depth = max(tmpl.depths(), default=0)
+        try:
+            w = dict(weights, mask_emb=weights["mask_emb"][:n].contiguous())
+            ctx = Bita(sh, w, tmpl, C_max=shape.prompt_len + (steps + 8) * (depth + 1) + rows + 64, device=dev)
+        except BitaError as e:
+            line.update(ms_per_step=None, refused=str(e))
+            print(json.dumps(line))
+            continue
+        ctx.prefill(prompt)
+        ms = _time_steps(ctx, steps)
         ctx.close()
+        line.update(ms_per_step=ms, tokens_per_s=acc / ms * 1e3, speedup_vs_autoregressive=(acc / ms) / (1.0 / ar_ms),
+                    weights_hbm_frac=shape.streamed_params * 2 / ms / 1e6 / peak)
+        print(json.dumps(line))
 
 
 def _spawn_ranks(n: int):

@@ -41,7 +41,7 @@ extern "C" {
 #define BITA_ERR_STATIC_SCRATCH (-8) /* problem needs more than the library's built-in scratch array  */
 
 #define BITA_MAX_NODES 160          /* tree nodes, root excluded                                      */
-#define BITA_MAX_ROWS 256           /* rows of the packed block: 1 + N + G * n_mask                   */
+#define BITA_MAX_ROWS 352           /* rows of the packed block: 1 + N + G * n_mask (a multiple of 32) */
 #define BITA_MAX_DEPTH 16
 #define BITA_MAX_TOPK 16            /* largest rank + 1 a template may use                            */
 #define BITA_MAX_MASK 8             /* mask tokens per group                                          */

@@ -10,7 +10,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libbita.so")
 
-MAX_NODES, MAX_ROWS, MAX_DEPTH, MAX_TOPK, MAX_MASK = 160, 256, 16, 16, 8
+MAX_NODES, MAX_ROWS, MAX_DEPTH, MAX_TOPK, MAX_MASK = 160, 352, 16, 16, 8
 
 
 class BitaError(RuntimeError):

@@ -333,14 +333,15 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
     const float sc = a.scale_log2;
     int gr[RT];
     bool row_live[RT], sees_p[RT];
-    uint32_t visw[RT][8];
+    constexpr int VW_MAX = BITA_MAX_ROWS / 32;                      // words of a row's ancestor bitmask
+    uint32_t visw[RT][VW_MAX];
     float m_run[RT], l_run[RT];
 #pragma unroll
     for (int t = 0; t < RT; ++t) {
       gr[t] = row0 + t * AU_ROWS + r;
       row_live[t] = gr[t] < a.M;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) {
+      for (int w = 0; w < VW_MAX; ++w) {
         visw[t][w] = (row_live[t] && w < a.W) ? a.vis[(size_t)b * a.vis_batch_stride + (size_t)gr[t] * a.W + w] : 0u;
         const int nb = a.M - 32 * w;                            // block rows this word can name
         if (nb < 32) visw[t][w] &= nb <= 0 ? 0u : ((1u << nb) - 1u);
@@ -384,7 +385,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
               const int q = j0 >= 0 ? j0 >> 5 : -1, sh = j0 & 31;
               uint32_t lo = q < 0 ? 0xffffffffu : 0u, hi = 0u;
 #pragma unroll
-              for (int u = 0; u < 8; ++u) {
+              for (int u = 0; u < VW_MAX; ++u) {
                 const uint32_t vw = second ? visw[RT - 1][u] : visw[0][u];
                 if (u == q) lo = vw;
                 if (u == q + 1) hi = vw;

@@ -387,7 +387,9 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc, g.a0, g.a1, map_b, p);
 }
 
-inline int pad16(int m) { return m <= 16 ? 16 : (m + 15) / 16 * 16; }
+// Padded row count of a block as the MMA sees it: a multiple of 16; past 256 rows a multiple of 32,
+// so that each of the two column halves is a multiple of 16.
+inline int pad16(int m) { return m <= 16 ? 16 : (m <= 256 ? (m + 15) / 16 * 16 : (m + 31) / 32 * 32); }
 
 // Attention launch shape: row tiles (one CTA takes one tile of 128 query rows, or two when the block
 // has more than 128 rows), and key slices.  The slices of a (sequence,
@@ -516,7 +518,7 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   auto it = c->act_maps.find(key);
   if (it == c->act_maps.end()) {
     CUtensorMap m;
-    int rc = make_map(&m, X, g.K, BITA_MAX_ROWS, n_pad);
+    int rc = make_map(&m, X, g.K, BITA_MAX_ROWS, n_pad > 256 ? n_pad / 2 : n_pad);
     if (rc) return rc;
     it = c->act_maps.emplace(key, m).first;
   }
@@ -1044,7 +1046,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   if ((rc = make_gemm_desc(&g, W, nullptr, N, K, 8))) return rc;
   const int n_pad = pad16(M);
   CUtensorMap mb;
-  if ((rc = make_map(&mb, X, K, M, n_pad))) return rc;
+  if ((rc = make_map(&mb, X, K, M, n_pad > 256 ? n_pad / 2 : n_pad))) return rc;
   const size_t cnt_bytes = align_up((size_t)g.tiles * 4);
   CU_TRY(cudaMemsetAsync(workspace, 0, ALIGN + cnt_bytes, s));     // status word and tile counters start at zero
   GemmTcParams p = epi_store((float*)Y, N);

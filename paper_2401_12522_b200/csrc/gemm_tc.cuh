@@ -1,6 +1,6 @@
 // Small-M weight-streaming projection on the 5th-generation tensor cores (sm_100a).
 //
-//   Y[m][n] = sum_k X[m][k] * W[n][k]      X: bf16 [M][K] (M <= 256 rows of the packed block)
+//   Y[m][n] = sum_k X[m][k] * W[n][k]      X: bf16 [M][K] (M <= BITA_MAX_ROWS rows of the packed block)
 //                                           W: bf16 [N][K] (a weight matrix, read exactly once)
 //
 // The roles are swapped with respect to a textbook GEMM: 128 weight rows are the MMA's M dimension
@@ -348,10 +348,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
           tma_load_2d(sa, &map_a0, kx, row_a, full, pol_w);
         }
       };
+      // the activation box holds at most 256 rows: larger blocks come as two boxes of n_pad / 2 rows
+      const int b_boxes = p.n_pad > 256 ? 2 : 1, b_rows = p.n_pad / b_boxes;
       auto load_b = [&](int i) {
         const int s = i % p.stages;
-        tma_load_2d(smem_base + (uint32_t)s * stage_bytes + a_bytes, &map_b, (kb0 + i) * TC_BLOCK_K, 0,
-                    smem_u32(&bar_full[s]), pol_x);
+        for (int h = 0; h < b_boxes; ++h)
+          tma_load_2d(smem_base + (uint32_t)s * stage_bytes + a_bytes + (uint32_t)(h * b_rows * TC_BLOCK_K * 2), &map_b,
+                      (kb0 + i) * TC_BLOCK_K, h * b_rows, smem_u32(&bar_full[s]), pol_x);
       };
       // Weights do not depend on earlier kernels: the first ring fill requests them before the
       // kernel waits for the producer of the activations.  One lane per stage issues that first
@@ -379,7 +382,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   } else if (warp == 1) {
     // ---------------- MMA issuer
     if (lane == 0 && nkb > 0) {
-      const uint32_t idesc = umma_idesc(p.n_pad);
+      // an MMA takes at most 256 columns: larger blocks are two column halves of n_pad / 2 (a multiple of 16)
+      const int halves = p.n_pad > 256 ? 2 : 1, n_half = p.n_pad / halves;
+      const uint32_t idesc = umma_idesc(n_half);
       bool ok = true;
       for (int i = 0; i < nkb && ok; ++i) {
         const int s = i % p.stages;
@@ -389,10 +394,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         tc_fence_after();
         const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
         const uint64_t da = umma_smem_desc(sa), db = umma_smem_desc(sa + a_bytes);
+        for (int h = 0; h < halves; ++h) {
+          // rows [h n_half, (h + 1) n_half) of the activation tile: n_half * 128 bytes further (n_half is a multiple of 8 rows)
+          const uint64_t dbh = db + (uint64_t)((h * n_half * TC_BLOCK_K * 2) >> 4);
 #pragma unroll
-        for (int k = 0; k < TC_BLOCK_K / TC_UMMA_K; ++k) {
-          // advancing 16 elements along K = 32 bytes = 2 units of the descriptor's address field
-          umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < TC_BLOCK_K / TC_UMMA_K; ++k) {
+            // advancing 16 elements along K = 32 bytes = 2 units of the descriptor's address field
+            umma_bf16(tmem_base + (uint32_t)(h * n_half), da + (uint64_t)(2 * k), dbh + (uint64_t)(2 * k), idesc,
+                      (i > 0 || k > 0) ? 1u : 0u);
+          }
         }
         umma_commit(smem_u32(&bar_empty[s]));                 // frees the stage when these MMAs are done
       }

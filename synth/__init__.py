@@ -11,9 +11,11 @@ from .model import CONFIGS, ModelShape, make_weights, layer_weight_specs  # noqa
 from .trees import (  # noqa: F401
     product_rule_template,
     comb_template,
+    full_tree_template,
     chain_template,
     random_recursive_template,
     empty_template,
     Template,
 )
 from .planting import plant_tree  # noqa: F401
+from .acceptance import AcceptanceModel, tokens_per_pass  # noqa: F401

@@ -70,6 +70,11 @@ def comb_template(n: int, k: int, *, per_node_groups: bool = True) -> Template:
     return Template(tuple(parent), tuple(rank), attach)
 
 
+def full_tree_template(n: int, k: int, *, per_node_groups: bool = True) -> Template:
+    """Fully tree-based decoding (Sec. 4.3, Table 4): every candidate of a depth has k children."""
+    return product_rule_template((k,) * n, (k ** n,) * n, per_node_groups=per_node_groups)
+
+
 def chain_template(n: int) -> Template:
     """Straightforward decoding (Sec. 3.2, Fig. 3): the top-1 draft of each mask, one group at the end."""
     return Template(tuple(range(-1, n - 1)), (0,) * n, (-1,))

@@ -71,10 +71,11 @@ def test_host_side_validation():
     # two groups on one attach point
     tm3, keep3 = _tmpl([-1], [0], [-1, -1])
     assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm3), shape.n_mask, C.byref(need)) == -2
-    # too many rows: 1 + 64 + 65 * 4 = 325 > 256
+    # a mask group on every node of the 64-node tree: 1 + 64 + 65 * 4 = 325 rows fit, 65 * 5 + 65 = 390 do not
     big = synth.product_rule_template((10, 6, 4, 2), (10, 6, 6, 4), per_node_groups=True)
     tm4, keep4 = _tmpl(big.parent, big.rank, big.attach)
-    assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm4), 4, C.byref(need)) == -2
+    assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm4), 4, C.byref(need)) == 0
+    assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm4), 5, C.byref(need)) == -2
     # rank beyond the top-k width
     tm5, keep5 = _tmpl([-1], [16], [-1])
     assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm5), shape.n_mask, C.byref(need)) == -2
@@ -83,6 +84,6 @@ def test_host_side_validation():
     assert lib.bita_step(None, None, None, C.byref(out)) == -1
     assert lib.bita_step_finish(None, C.byref(out)) == -1
     assert lib.bita_strerror(-3) == b"KV cache full"
-    assert lib.bita_gemm_workspace_bytes(300, 8, 8, C.byref(need)) == -1
+    assert lib.bita_gemm_workspace_bytes(400, 8, 8, C.byref(need)) == -1
     assert lib.bita_gemm_workspace_bytes(4, 8, 12, C.byref(need)) == -1
     assert lib.bita_attention_workspace_bytes(1, 19, 4, 96, C.byref(need)) == -1

@@ -23,7 +23,8 @@ def test_generators_are_bit_identical_on_cpu_and_gpu():
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (19, 1376, 256), (19, 256, 688), (69, 1000, 4096),
                                    (133, 384, 1024), (256, 130, 520), (105, 4096, 4096), (128, 4096, 2048),
-                                   (154, 4096, 4096), (200, 1000, 11008), (256, 12288, 4096)])
+                                   (154, 4096, 4096), (200, 1000, 11008), (256, 12288, 4096),
+                                   (260, 1000, 512), (325, 4096, 4096), (340, 300, 11008), (352, 12288, 4096)])
 def test_projection_matches_fp64_matmul(M, N, K):
     from paper_2401_12522_b200 import bita_gemm_bf16
     X = synth.pseudo_normal(3, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda:0")
@@ -78,7 +79,7 @@ def check_attention_against_oracle(out, q, k, v, pk, pv, ctx, blk, H_kv, P):
 
 
 ATTENTION_CASES = [(1, 16, 4, 4, 64, 16, 70), (2, 16, 8, 2, 128, 16, 300), (1, 64, 4, 4, 128, 0, 513),
-                   (1, 128, 2, 1, 128, 5, 40), (1, 0, 4, 2, 64, 16, 0)]
+                   (1, 128, 2, 1, 128, 5, 40), (1, 0, 4, 2, 64, 16, 0), (1, 158, 4, 2, 128, 16, 200)]
 
 
 @pytest.mark.parametrize("B,N,H,H_kv,D,P,C", ATTENTION_CASES)
@@ -112,10 +113,10 @@ def test_tree_attention_workspace_route_matches_oracle(B, N, H, H_kv, D, P, C):
 
 # ------------------------------------------------------------------ the whole pass, lockstep
 
-@pytest.mark.parametrize("plen", [1, 140, 300])
+@pytest.mark.parametrize("plen", [1, 140, 300, 700])
 def test_first_pass_in_several_blocks(plen):
-    """Prompts longer than one block of the first pass (248 query rows): 140 tokens make one block of
-    143 rows (past 128: two attention row tiles), 300 make two blocks of 150."""
+    """First passes of several shapes: 140 tokens make one block of 143 rows (past 128: two attention
+    row tiles), 300 one block of 303 rows (past 256: two MMA column halves), 700 three blocks of 234."""
     shape = synth.CONFIGS["tiny"]
     tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
     seed = 0x5EED0777
@@ -140,7 +141,10 @@ TEMPLATES = {
     "comb-n3k5-pernode": (lambda: synth.comb_template(3, 5), 3),
     "comb-n4k3-pernode": (lambda: synth.comb_template(4, 3), 4),
     "comb-n4k5-pernode": (lambda: synth.comb_template(4, 5), 4),     # 105 rows: past 96, one row tile
-    "comb-n4k12-pernode": (lambda: synth.comb_template(4, 12), 4),   # 245 rows: near the limit, two row tiles
+    "comb-n4k12-pernode": (lambda: synth.comb_template(4, 12), 4),   # 245 rows: two attention row tiles
+    # past 256 rows: two MMA column halves in the projections, a second attention CTA per head
+    "product64-pernode": (lambda: synth.product_rule_template((10, 6, 4, 2), (10, 6, 6, 4), per_node_groups=True), 4),  # 325 rows
+    "full-n3k4-pernode": (lambda: synth.full_tree_template(3, 4), 3),   # 340 rows
     "chain": (lambda: synth.chain_template(3), 3),
     "empty": (lambda: synth.empty_template(), 3),
     "product-pernode": (lambda: synth.product_rule_template((3, 3, 3), (3, 3, 3), per_node_groups=True), 3),
@@ -390,14 +394,20 @@ def _write_report(ls):
 
 
 @pytest.mark.parametrize("name,layers,prompt_len,comb", [("7b", 2, 150, False), ("13b", 1, 140, False),
-                                                         ("70b", 1, 70, False), ("7b", 1, 120, True)])
+                                                         ("70b", 1, 70, False), ("7b", 1, 120, True),
+                                                         ("7b", 1, 300, "pernode64")])
 def test_full_width_shapes_lockstep(name, layers, prompt_len, comb):
     """Model width, head layout, FFN width, vocabulary, tree and block size of the measured configs;
     only the depth is cut so that the fp64 oracle finishes in seconds.  Every kernel runs in the
     grid/cluster/tile configuration of the full-depth step (none depends on the layer count)."""
     shape = synth.CONFIGS[name].with_layers(layers)
     # comb: the paper's default tree (k = 5 candidates per depth, a mask group per node): 105 rows
-    tmpl = synth.comb_template(shape.n_mask, 5) if comb else synth.product_rule_template(shape.tree_K, shape.tree_B)
+    if comb == "pernode64":
+        # the paper's method on the measured 64-node tree: a mask group on every node, 325 rows; the
+        # 300-token prompt makes the first pass one block of 304 rows
+        tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B, per_node_groups=True)
+    else:
+        tmpl = synth.comb_template(shape.n_mask, 5) if comb else synth.product_rule_template(shape.tree_K, shape.tree_B)
     seed = 0x5EED0010
     prompt = prompt_tokens(seed, prompt_len, shape.V)
     ref_model = oracle_model(shape, seed, lazy=True)
