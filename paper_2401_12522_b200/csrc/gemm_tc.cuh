@@ -282,6 +282,230 @@ __device__ __forceinline__ void tmem_st64(uint32_t taddr, const float* v) {
       : "memory");
 }
 // ---------------------------------------------------------------------------------------------
+// Fused operation of a projection on rows [t0, t0 + cnt) of a tile, by all warps of the CTA.  A
+// thread handles 4 consecutive features (quad = lane) of one row at a time; the warps take rows
+// round-robin, RB rows of a warp per batch so that their loads fly together.  Partner features of
+// the rotary embedding and of SwiGLU sit 64 (or 32) features away, i.e. 16 (or 8) lanes, and are
+// exchanged with a warp shuffle.
+//   SU == 0: the tile is complete in shared memory (`recv`, row-major [cnt][128] fp32).
+//   SU  > 0: the tile is the sum of p.splits partial tiles in the exchange buffer (`part_tile`,
+//            split-major).  A thread first requests everything that does not depend on the other
+//            splits (residual rows, rotary factors), then `all_in()` (called by every thread of the
+//            CTA, exactly once) waits for the splits, then the thread sums its quads over the
+//            partial tiles, always in split order, SU loads per row in flight.
+template <int RB, int SU, typename AllIn>
+__device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const float* recv, const float* part_tile,
+                                               size_t tile_elems, const float* rstd_s, int tile, int n_tiles, int t0,
+                                               int cnt, int warp, int lane, AllIn all_in) {
+  constexpr int NW = TC_THREADS / 32;
+  const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
+  const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
+  float g4[4] = {1.f, 1.f, 1.f, 1.f};
+  if (p.mode == EPI_RESID && n4 + 3 < p.N) {
+    const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
+    g4[0] = a.x; g4[1] = a.y; g4[2] = b.x; g4[3] = b.y;
+  }
+  // EPI_QKV: which head this quad belongs to
+  const int half = p.mode == EPI_QKV ? p.D >> 1 : 2;
+  const int sh = half >> 2;                                  // partner quad is `sh` lanes away (16 or 8)
+  const int head = p.mode == EPI_QKV ? n4 / p.D : 0, dd = p.mode == EPI_QKV ? n4 - head * p.D : 0;
+  const bool lo = dd < half;
+  const int jr = lo ? dd : dd - half;
+  const bool rot = p.mode == EPI_QKV && n4 < p.N && head < p.H + p.H_kv;
+  const bool in_n = n4 + 3 < p.N;
+  const float sg = lo ? -1.f : 1.f;
+
+  // every warp runs the same number of batches (the wait below holds a CTA-wide barrier)
+  for (int b0 = 0; b0 < cnt || (SU > 0 && b0 == 0); b0 += NW * RB) {
+    const int tb = b0 + warp;
+    // phase A: every load of the batch (global operands, partial sums, row scales)
+    float4 g0[RB], g1[RB], acc[RB];
+    float rs[RB];
+    bool live[RB];
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int tl = tb + NW * u;
+      live[u] = tl < cnt;
+      const int tlc = live[u] ? tl : (tb < cnt ? tb : 0);    // clamp: dead rows recompute a live row, store nothing
+      const int tok = t0 + tlc;
+      g0[u] = make_float4(1.f, 0.f, 1.f, 0.f);
+      g1[u] = make_float4(1.f, 0.f, 1.f, 0.f);
+      if (cnt > 0) {
+        if (p.mode == EPI_RESID) {
+          if (in_n) g0[u] = *reinterpret_cast<const float4*>(p.x + (size_t)tok * p.N + n4);
+        } else if (rot) {
+          g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
+          g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
+        }
+      }
+      rs[u] = cnt > 0 ? rstd_s[tok] : 0.f;
+    }
+    if constexpr (SU > 0) {
+      if (b0 == 0) all_in();
+#pragma unroll
+      for (int u = 0; u < RB; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s0 = 0; s0 < p.splits; s0 += SU) {
+        float4 v[RB][SU];
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          const float4* src = reinterpret_cast<const float4*>(part_tile + (size_t)(t0 + tb + NW * u) * TC_BLOCK_N) + lane;
+#pragma unroll
+          for (int r = 0; r < SU; ++r)
+            if (live[u] && s0 + r < p.splits) v[u][r] = __ldcg(src + (size_t)(s0 + r) * (tile_elems / 4));
+        }
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+#pragma unroll
+          for (int r = 0; r < SU; ++r)
+            if (live[u] && s0 + r < p.splits) {
+              acc[u].x += v[u][r].x; acc[u].y += v[u][r].y; acc[u].z += v[u][r].z; acc[u].w += v[u][r].w;
+            }
+        }
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        const int tlc = live[u] ? tb + NW * u : (tb < cnt ? tb : 0);
+        acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < RB; ++u) { acc[u].x *= rs[u]; acc[u].y *= rs[u]; acc[u].z *= rs[u]; acc[u].w *= rs[u]; }
+
+    // phase B: the fused operation, written batch-wide so that independent rows interleave
+    if (p.mode == EPI_RESID) {
+      float ss[RB];
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        ss[u] = 0.f;
+        if (in_n) {                                          // N (the model width) is a multiple of 8
+          float4 xv = g0[u];
+          xv.x += acc[u].x; xv.y += acc[u].y; xv.z += acc[u].z; xv.w += acc[u].w;
+          ss[u] = live[u] ? xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w : 0.f;
+          if (live[u]) {
+            const int tok = t0 + tb + NW * u;
+            *reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4) = xv;
+            uint2 pk;
+            pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
+            pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
+            *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
+          }
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int u = 0; u < RB; ++u) ss[u] += __shfl_xor_sync(0xffffffffu, ss[u], o);
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int u = 0; u < RB; ++u)
+          if (live[u]) atomicAdd(p.out_sumsq + t0 + tb + NW * u, sumsq_to_fixed(ss[u]));
+      }
+    } else if (p.mode == EPI_STORE || p.mode == EPI_HEAD) {
+      if (p.mode == EPI_HEAD) {
+        // Per row: the best entries of this tile, picked one at a time by a warp-wide maximum over
+        // ordered keys (a key is unique, so "remove the winner" is an equality test).
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          if (!live[u]) continue;                              // warp-uniform
+          const int row = t0 + tb + NW * u;
+          const int kk = p.row_kind[row] == ROW_MASK ? p.k_max : 1;
+          unsigned long long key[4];
+          const float vals[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) key[e] = n4 + e < p.N ? select_key(vals[e], n4 + e) : 0ull;
+          unsigned long long* dst = p.cand + ((size_t)row * n_tiles + tile) * BITA_MAX_TOPK;
+          for (int t = 0; t < kk; ++t) {
+            unsigned long long best = max(max(key[0], key[1]), max(key[2], key[3]));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (key[e] == best) key[e] = 0ull;
+            if (lane == 0) dst[t] = best;
+          }
+        }
+        if (!p.out) continue;
+      }
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        if (!live[u]) continue;
+        float* dst = p.out + (size_t)(t0 + tb + NW * u) * p.ldo + n4;
+        if (in_n && (p.ldo & 3) == 0) {
+          *reinterpret_cast<float4*>(dst) = acc[u];
+        } else {
+          if (n4 < p.N) dst[0] = acc[u].x;
+          if (n4 + 1 < p.N) dst[1] = acc[u].y;
+          if (n4 + 2 < p.N) dst[2] = acc[u].z;
+          if (n4 + 3 < p.N) dst[3] = acc[u].w;
+        }
+      }
+    } else if (p.mode == EPI_SWIGLU) {
+      // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
+      float4 up[RB];
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        up[u].x = __shfl_down_sync(0xffffffffu, acc[u].x, 16);
+        up[u].y = __shfl_down_sync(0xffffffffu, acc[u].y, 16);
+        up[u].z = __shfl_down_sync(0xffffffffu, acc[u].z, 16);
+        up[u].w = __shfl_down_sync(0xffffffffu, acc[u].w, 16);
+      }
+      const int f = tile * 64 + 4 * lane;
+      if (lane < 16 && f < p.F) {                            // F is a multiple of 8: a quad is all in or all out
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          const float h0 = __fdividef(acc[u].x, 1.0f + __expf(-acc[u].x)) * up[u].x;
+          const float h1 = __fdividef(acc[u].y, 1.0f + __expf(-acc[u].y)) * up[u].y;
+          const float h2 = __fdividef(acc[u].z, 1.0f + __expf(-acc[u].z)) * up[u].z;
+          const float h3 = __fdividef(acc[u].w, 1.0f + __expf(-acc[u].w)) * up[u].w;
+          uint2 pk;
+          pk.x = pack_bf16x2(h0, h1);
+          pk.y = pack_bf16x2(h2, h3);
+          if (live[u]) *reinterpret_cast<uint2*>(p.hf + (size_t)(t0 + tb + NW * u) * p.F + f) = pk;
+        }
+      }
+    } else {                                                 // EPI_QKV
+      // partner values: the other half of the same head
+      float4 w[RB];
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        w[u].x = __shfl_xor_sync(0xffffffffu, acc[u].x, sh);
+        w[u].y = __shfl_xor_sync(0xffffffffu, acc[u].y, sh);
+        w[u].z = __shfl_xor_sync(0xffffffffu, acc[u].z, sh);
+        w[u].w = __shfl_xor_sync(0xffffffffu, acc[u].w, sh);
+      }
+      if (n4 < p.N) {                                        // N is a multiple of D: a quad is all in or all out
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+          float4 r = acc[u];
+          if (rot) {
+            r.x = acc[u].x * g0[u].x + sg * w[u].x * g0[u].y;
+            r.y = acc[u].y * g0[u].z + sg * w[u].y * g0[u].w;
+            r.z = acc[u].z * g1[u].x + sg * w[u].z * g1[u].y;
+            r.w = acc[u].w * g1[u].z + sg * w[u].w * g1[u].w;
+          }
+          uint2 pk;
+          pk.x = pack_bf16x2(r.x, r.y);
+          pk.y = pack_bf16x2(r.z, r.w);
+          if (!live[u]) continue;
+          const int tok = t0 + tb + NW * u;
+          const int slot = C + tok;
+          if (head < p.H) {
+            *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
+          } else if (slot < p.C_max) {
+            bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
+                                             : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
+            *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
+          }
+        }
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
           const __grid_constant__ CUtensorMap map_b, GemmTcParams p) {
@@ -454,253 +678,47 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   }
   tc_fence_before();
   __syncthreads();
+  // ---------------- epilogue, part 2: reduction over the splits + fused operation, all six warps.
   // Rows of the tile this CTA finishes: all of them without a split, else an equal share, so that
   // the reduction and the fused operation of a tile are spread over all its splits.
   const int t0 = p.splits > 1 ? (int)((long)p.M * split / p.splits) : 0;
   const int cnt = (p.splits > 1 ? (int)((long)p.M * (split + 1) / p.splits) : p.M) - t0;
-  if (p.splits > 1) {
+  pdl_wait();
+  if (p.splits == 1) {
+    fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, [] {});
+  } else {
     int32_t* arrived = p.tile_counters + tile;
     int32_t* departed = p.tile_counters + TC_DEPART_OFFSET + tile;
     if (threadIdx.x == 0) {
-      // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
-      // before it has published its own partial tile: the wait ends, and it is bounded all the same.
       __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
       atomicAdd(arrived, 1);
-      unsigned long long w0 = 0;
-      bool ok = true;
-      for (uint32_t spin = 0; ld_acquire_gpu(arrived) < p.splits; ++spin) {
-        if ((spin & 63u) == 63u) {
-          const unsigned long long now = global_ns();
-          if (w0 == 0) w0 = now;
-          else if (now - w0 > p.wait_ns) { ok = false; break; }
-        }
-      }
-      if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
-      __threadfence();
     }
-    __syncthreads();
-    // Sum rows t0 .. t0+cnt of the partial tiles into `stg` (local row order), in split order.  A
-    // thread takes 16-byte items; the loads of four items (four splits each) fly together.
-    const int items = cnt * (TC_BLOCK_N / 4);
-    const float4* src = reinterpret_cast<const float4*>(part_tile) + (size_t)t0 * (TC_BLOCK_N / 4);
-    const int stride4 = (int)(tile_elems / 4);               // between the splits' tiles
-    for (int i0 = threadIdx.x; i0 < items; i0 += 4 * TC_THREADS) {
-      float4 a4[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) a4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int r0 = 0; r0 < p.splits; r0 += 4) {
-        float4 v[4][4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = min(i0 + u * TC_THREADS, items - 1);
-#pragma unroll
-          for (int r = 0; r < 4; ++r)
-            if (r0 + r < p.splits) v[u][r] = __ldcg(src + (size_t)(r0 + r) * stride4 + i);
+    // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
+    // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+    auto all_in = [&]() {
+      if (threadIdx.x == 0) {
+        unsigned long long w0 = 0;
+        bool ok = true;
+        for (uint32_t spin = 0; ld_acquire_gpu(arrived) < p.splits; ++spin) {
+          if ((spin & 63u) == 63u) {
+            const unsigned long long now = global_ns();
+            if (w0 == 0) w0 = now;
+            else if (now - w0 > p.wait_ns) { ok = false; break; }
+          }
         }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-#pragma unroll
-          for (int r = 0; r < 4; ++r)
-            if (r0 + r < p.splits) { a4[u].x += v[u][r].x; a4[u].y += v[u][r].y; a4[u].z += v[u][r].z; a4[u].w += v[u][r].w; }
-        }
+        if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
+        __threadfence();
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * TC_THREADS;
-        if (i < items) reinterpret_cast<float4*>(stg)[i] = a4[u];
-      }
-    }
+      __syncthreads();
+    };
+    if (p.splits <= 4) fused_epilogue<4, 4>(p, nullptr, part_tile, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, all_in);
+    else fused_epilogue<2, 8>(p, nullptr, part_tile, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, all_in);
     __syncthreads();
     // The partial tiles are read: the last split to say so leaves both counters at zero for the
     // next projection (which touches them only after this kernel has completed).
     if (threadIdx.x == 0) {
       const int old = atomicAdd(departed, 1);
       if (old == p.splits - 1) { *arrived = 0; *departed = 0; }
-    }
-  }
-  const float* recv = stg;
-
-  // ---------------- epilogue, part 2: reduction over the splits + fused operation, all six warps.
-  // A thread handles 4 consecutive features (quad = lane) of one row at a time; the warps take
-  // rows round-robin.  Partner features of the rotary embedding and of SwiGLU sit 64 (or 32)
-  // features away, i.e. 16 (or 8) lanes, and are exchanged with a warp shuffle.
-  {
-    constexpr int RB = 6;                                      // rows per batch: their global loads fly together
-    constexpr int NW = TC_THREADS / 32;
-    pdl_wait();
-    const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
-    const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
-    float g4[4] = {1.f, 1.f, 1.f, 1.f};
-    if (p.mode == EPI_RESID && n4 + 3 < p.N) {
-      const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
-      const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.x));
-      const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
-      g4[0] = a.x; g4[1] = a.y; g4[2] = b.x; g4[3] = b.y;
-    }
-    // EPI_QKV: which head this quad belongs to
-    const int half = p.mode == EPI_QKV ? p.D >> 1 : 2;
-    const int sh = half >> 2;                                  // partner quad is `sh` lanes away (16 or 8)
-    const int head = p.mode == EPI_QKV ? n4 / p.D : 0, dd = p.mode == EPI_QKV ? n4 - head * p.D : 0;
-    const bool lo = dd < half;
-    const int jr = lo ? dd : dd - half;
-    const bool rot = p.mode == EPI_QKV && n4 < p.N && head < p.H + p.H_kv;
-    const bool in_n = n4 + 3 < p.N;
-    const float sg = lo ? -1.f : 1.f;
-
-    for (int tb = warp; tb < cnt; tb += NW * RB) {
-      // phase A: every load of the batch (global operands, partial sums, row scales)
-      float4 g0[RB], g1[RB], acc[RB];
-      float rs[RB];
-      bool live[RB];
-#pragma unroll
-      for (int u = 0; u < RB; ++u) {
-        const int tl = tb + NW * u;
-        live[u] = tl < cnt;
-        const int tlc = live[u] ? tl : tb;                     // clamp: dead rows recompute row tb, store nothing
-        const int tok = t0 + tlc;
-        g0[u] = make_float4(1.f, 0.f, 1.f, 0.f);
-        g1[u] = make_float4(1.f, 0.f, 1.f, 0.f);
-        if (p.mode == EPI_RESID) {
-          if (in_n) g0[u] = *reinterpret_cast<const float4*>(p.x + (size_t)tok * p.N + n4);
-        } else if (rot) {
-          g0[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr);
-          g1[u] = *reinterpret_cast<const float4*>(p.rope_blk + (size_t)tok * half + jr + 2);
-        }
-        acc[u] = *reinterpret_cast<const float4*>(recv + (size_t)tlc * TC_BLOCK_N + 4 * lane);
-        rs[u] = rstd_s[t0 + tlc];
-      }
-#pragma unroll
-      for (int u = 0; u < RB; ++u) { acc[u].x *= rs[u]; acc[u].y *= rs[u]; acc[u].z *= rs[u]; acc[u].w *= rs[u]; }
-
-      // phase B: the fused operation, written batch-wide so that independent rows interleave
-      if (p.mode == EPI_RESID) {
-        float ss[RB];
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-          ss[u] = 0.f;
-          if (in_n) {                                          // N (the model width) is a multiple of 8
-            float4 xv = g0[u];
-            xv.x += acc[u].x; xv.y += acc[u].y; xv.z += acc[u].z; xv.w += acc[u].w;
-            ss[u] = live[u] ? xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w : 0.f;
-            if (live[u]) {
-              const int tok = t0 + tb + NW * u;
-              *reinterpret_cast<float4*>(p.x + (size_t)tok * p.N + n4) = xv;
-              uint2 pk;
-              pk.x = pack_bf16x2(xv.x * g4[0], xv.y * g4[1]);
-              pk.y = pack_bf16x2(xv.z * g4[2], xv.w * g4[3]);
-              *reinterpret_cast<uint2*>(p.xhat + (size_t)tok * p.N + n4) = pk;
-            }
-          }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-          for (int u = 0; u < RB; ++u) ss[u] += __shfl_xor_sync(0xffffffffu, ss[u], o);
-        }
-        if (lane == 0) {
-#pragma unroll
-          for (int u = 0; u < RB; ++u)
-            if (live[u]) atomicAdd(p.out_sumsq + t0 + tb + NW * u, sumsq_to_fixed(ss[u]));
-        }
-      } else if (p.mode == EPI_STORE || p.mode == EPI_HEAD) {
-        if (p.mode == EPI_HEAD) {
-          // Per row: the best entries of this tile, picked one at a time by a warp-wide maximum over
-          // ordered keys (a key is unique, so "remove the winner" is an equality test).
-#pragma unroll
-          for (int u = 0; u < RB; ++u) {
-            if (!live[u]) continue;                              // warp-uniform
-            const int row = t0 + tb + NW * u;
-            const int kk = p.row_kind[row] == ROW_MASK ? p.k_max : 1;
-            unsigned long long key[4];
-            const float vals[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) key[e] = n4 + e < p.N ? select_key(vals[e], n4 + e) : 0ull;
-            unsigned long long* dst = p.cand + ((size_t)row * gridDim.x + tile) * BITA_MAX_TOPK;
-            for (int t = 0; t < kk; ++t) {
-              unsigned long long best = max(max(key[0], key[1]), max(key[2], key[3]));
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (key[e] == best) key[e] = 0ull;
-              if (lane == 0) dst[t] = best;
-            }
-          }
-          if (!p.out) continue;
-        }
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-          if (!live[u]) continue;
-          float* dst = p.out + (size_t)(t0 + tb + NW * u) * p.ldo + n4;
-          if (in_n && (p.ldo & 3) == 0) {
-            *reinterpret_cast<float4*>(dst) = acc[u];
-          } else {
-            if (n4 < p.N) dst[0] = acc[u].x;
-            if (n4 + 1 < p.N) dst[1] = acc[u].y;
-            if (n4 + 2 < p.N) dst[2] = acc[u].z;
-            if (n4 + 3 < p.N) dst[3] = acc[u].w;
-          }
-        }
-      } else if (p.mode == EPI_SWIGLU) {
-        // lanes 0..15 hold gate features 4*lane.., lanes 16..31 the matching up features
-        float4 up[RB];
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-          up[u].x = __shfl_down_sync(0xffffffffu, acc[u].x, 16);
-          up[u].y = __shfl_down_sync(0xffffffffu, acc[u].y, 16);
-          up[u].z = __shfl_down_sync(0xffffffffu, acc[u].z, 16);
-          up[u].w = __shfl_down_sync(0xffffffffu, acc[u].w, 16);
-        }
-        const int f = tile * 64 + 4 * lane;
-        if (lane < 16 && f < p.F) {                            // F is a multiple of 8: a quad is all in or all out
-#pragma unroll
-          for (int u = 0; u < RB; ++u) {
-            const float h0 = __fdividef(acc[u].x, 1.0f + __expf(-acc[u].x)) * up[u].x;
-            const float h1 = __fdividef(acc[u].y, 1.0f + __expf(-acc[u].y)) * up[u].y;
-            const float h2 = __fdividef(acc[u].z, 1.0f + __expf(-acc[u].z)) * up[u].z;
-            const float h3 = __fdividef(acc[u].w, 1.0f + __expf(-acc[u].w)) * up[u].w;
-            uint2 pk;
-            pk.x = pack_bf16x2(h0, h1);
-            pk.y = pack_bf16x2(h2, h3);
-            if (live[u]) *reinterpret_cast<uint2*>(p.hf + (size_t)(t0 + tb + NW * u) * p.F + f) = pk;
-          }
-        }
-      } else {                                                 // EPI_QKV
-        // partner values: the other half of the same head
-        float4 w[RB];
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-          w[u].x = __shfl_xor_sync(0xffffffffu, acc[u].x, sh);
-          w[u].y = __shfl_xor_sync(0xffffffffu, acc[u].y, sh);
-          w[u].z = __shfl_xor_sync(0xffffffffu, acc[u].z, sh);
-          w[u].w = __shfl_xor_sync(0xffffffffu, acc[u].w, sh);
-        }
-        if (n4 < p.N) {                                        // N is a multiple of D: a quad is all in or all out
-#pragma unroll
-          for (int u = 0; u < RB; ++u) {
-            float4 r = acc[u];
-            if (rot) {
-              r.x = acc[u].x * g0[u].x + sg * w[u].x * g0[u].y;
-              r.y = acc[u].y * g0[u].z + sg * w[u].y * g0[u].w;
-              r.z = acc[u].z * g1[u].x + sg * w[u].z * g1[u].y;
-              r.w = acc[u].w * g1[u].z + sg * w[u].w * g1[u].w;
-            }
-            uint2 pk;
-            pk.x = pack_bf16x2(r.x, r.y);
-            pk.y = pack_bf16x2(r.z, r.w);
-            if (!live[u]) continue;
-            const int tok = t0 + tb + NW * u;
-            const int slot = C + tok;
-            if (head < p.H) {
-              *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
-            } else if (slot < p.C_max) {
-              bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
-                                               : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
-              *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
-            }
-          }
-        }
-      }
     }
   }
   __syncthreads();
