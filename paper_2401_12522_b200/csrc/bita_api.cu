@@ -273,12 +273,16 @@ struct GemmDesc {
   CUtensorMap a0, a1;
   const void *w0 = nullptr, *w1 = nullptr;
   int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
+  int kind = 0;           // which set of split-arrival counters its launches count on (GemmKind)
 };
 
 // Split-K factor: as many CTAs as stay resident together (two per SM while the block is small, the
 // shared-memory ring of a CTA then being half an SM's), never fewer than 4 K blocks per split.
 constexpr int GEMM_MAX_CTAS = 296;       // size of the exchange buffer: two CTAs on each of up to 148 SMs
 constexpr int GEMM_MAX_SPLITS = 8;
+// Launches that may follow one another with different shapes count their split arrivals on sets of
+// their own, so that every counter of a set moves by the same amount with every launch of its kind.
+enum GemmKind { KIND_QKV = 0, KIND_O, KIND_GU, KIND_DN, KIND_HEAD, GEMM_KINDS };
 
 // What the library remembers per device of the process: CUDA keeps function attributes and
 // device properties per device, so none of this may be a process-wide flag.
@@ -342,6 +346,7 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
     if ((rc = make_map(&g->a0, W0, K, N, TC_BLOCK_N))) return rc;
     g->a1 = g->a0;
   }
+  if (g->tiles > TC_MAX_TILES) return BITA_ERR_INVALID_ARG;
   g->splits = gemm_splits(g->tiles, K, max_splits);
   return BITA_OK;
 }
@@ -446,7 +451,7 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
   t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
-  t.gemm_cnt = (int32_t*)take(4096 * 4);
+  t.gemm_cnt = (int32_t*)take((size_t)GEMM_KINDS * TC_MAX_TILES * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState));
@@ -479,6 +484,7 @@ struct bita_ctx {
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
   std::map<std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>, AttnMaps> attn_map_cache;
   bool pdl;                             // programmatic dependent launch between the kernels of a pass
+  uint32_t split_arrivals[GEMM_KINDS];  // what every counter of a set has reached once the launches so far are done
   unsigned long long wait_ns;           // bound of every device-side wait
   int last_rows;                        // rows of the most recent pass (what the debug buffer holds)
 
@@ -525,7 +531,12 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   p.status = &c->b.state->status;
   p.wait_ns = c->wait_ns;
   p.part = c->b.gemm_part;
-  p.tile_counters = c->b.gemm_cnt;
+  p.tile_counters = c->b.gemm_cnt + (size_t)g.kind * TC_MAX_TILES;
+  {
+    const int splits = effective_splits(g, n_pad);
+    if (splits > 1) c->split_arrivals[g.kind] += (uint32_t)splits;
+    p.arrive_target = (int32_t)c->split_arrivals[g.kind];
+  }
   mark(c, 0);
   int rc = launch_gemm_tc(g, it->second, n_pad, M, p, c->pdl, c->stream);
   c->launches++;
@@ -814,12 +825,15 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
       if ((rc = make_gemm_desc(&c->d_o[l], c->wo[l], nullptr, dims->d, dims->H * dims->D, 8))) return fail(rc);
       if ((rc = make_gemm_desc(&c->d_gu[l], c->wg[l], c->wu[l], dims->F, dims->d, 8))) return fail(rc);
       if ((rc = make_gemm_desc(&c->d_dn[l], c->wd[l], nullptr, dims->d, dims->F, 8))) return fail(rc);
+      c->d_qkv[l].kind = KIND_QKV; c->d_o[l].kind = KIND_O; c->d_gu[l].kind = KIND_GU; c->d_dn[l].kind = KIND_DN;
     }
     if ((rc = make_gemm_desc(&c->d_head, c->lm_head, nullptr, dims->V, dims->d, 1))) return fail(rc);
+    c->d_head.kind = KIND_HEAD;
   }
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
-  if (cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  if (cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
@@ -829,7 +843,8 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
 int bita_reset(bita_ctx* c, bita_kv* kv) {
   if (!c || !kv) return BITA_ERR_INVALID_ARG;
   // a pass that gave up on a wait may have left split counters half way
-  CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, 4096 * 4, c->stream));
+  CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream));
+  for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
   k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
   CU_TRY(cudaStreamSynchronize(c->stream));
   c->prefilled = false;
@@ -1053,6 +1068,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   p.status = (int32_t*)workspace;
   p.tile_counters = (int32_t*)((uint8_t*)workspace + ALIGN);
   p.part = (float*)((uint8_t*)workspace + ALIGN + cnt_bytes);
+  p.arrive_target = effective_splits(g, n_pad);                    // the counters were just cleared
   if ((rc = launch_gemm_tc(g, mb, n_pad, M, p, false, s))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;

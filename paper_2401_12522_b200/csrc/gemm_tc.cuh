@@ -37,7 +37,7 @@ constexpr int TC_BLOCK_N = 128;   // weight rows per tile (MMA M)
 constexpr int TC_BLOCK_K = 64;    // bf16 elements per K block = 128 bytes = one swizzle row
 constexpr int TC_UMMA_K = 16;
 constexpr int TC_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
-constexpr int TC_DEPART_OFFSET = 2048;     // tile_counters: [0, 2048) arrivals, [2048, 4096) departures
+constexpr int TC_MAX_TILES = 2048;          // tiles a launch with split-K may have (one arrival counter each)
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // default bound of a device-side wait: 2 s
 
 enum GemmEpilogue : int32_t {
@@ -93,7 +93,8 @@ struct GemmTcParams {
   int32_t* status;       // device status word (sticky error flag)
   unsigned long long wait_ns;   // bound of every device-side wait of the launch
   float* part;           // split-K exchange buffer [tiles][splits][M][128] fp32 (splits > 1)
-  int32_t* tile_counters;  // [4096]: arrivals per tile, then (at TC_DEPART_OFFSET) departures; zero before the launch, left zero
+  int32_t* tile_counters;  // [tiles] arrivals per tile; they only ever count up: a launch adds `splits` to each of them
+  int32_t arrive_target;   // value of a tile's counter once all splits of THIS launch are in (wraps; compared as a difference)
   // row scale of the input (RMSNorm statistics of the rows of X), or null: y *= rstd(row)
   const unsigned long long* in_sumsq;
   int32_t norm_d;
@@ -688,18 +689,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, [] {});
   } else {
     int32_t* arrived = p.tile_counters + tile;
-    int32_t* departed = p.tile_counters + TC_DEPART_OFFSET + tile;
     if (threadIdx.x == 0) {
       __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
       atomicAdd(arrived, 1);
     }
     // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
     // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+    // The counter is never reset: the host tells each launch the value that means "all in", so no
+    // split has to report that it has finished reading (the exchange buffer is next written by a
+    // later kernel, which starts its own stores only after this one has completed).
     auto all_in = [&]() {
       if (threadIdx.x == 0) {
         unsigned long long w0 = 0;
         bool ok = true;
-        for (uint32_t spin = 0; ld_acquire_gpu(arrived) < p.splits; ++spin) {
+        for (uint32_t spin = 0; (int32_t)((uint32_t)ld_acquire_gpu(arrived) - (uint32_t)p.arrive_target) < 0; ++spin) {
           if ((spin & 63u) == 63u) {
             const unsigned long long now = global_ns();
             if (w0 == 0) w0 = now;
@@ -711,15 +714,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
       }
       __syncthreads();
     };
-    if (p.splits <= 4) fused_epilogue<4, 4>(p, nullptr, part_tile, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, all_in);
-    else fused_epilogue<2, 8>(p, nullptr, part_tile, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, all_in);
-    __syncthreads();
-    // The partial tiles are read: the last split to say so leaves both counters at zero for the
-    // next projection (which touches them only after this kernel has completed).
-    if (threadIdx.x == 0) {
-      const int old = atomicAdd(departed, 1);
-      if (old == p.splits - 1) { *arrived = 0; *departed = 0; }
-    }
+    // rows per batch x loads per row in flight, sized so that a 69..128-row block takes one batch
+    const int nt = (int)gridDim.x;
+    if (p.splits == 2) fused_epilogue<6, 2>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+    else if (p.splits == 3) fused_epilogue<4, 3>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+    else if (p.splits == 4) fused_epilogue<4, 4>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+    else fused_epilogue<2, 8>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
   }
   __syncthreads();
   if (warp == 1) {
