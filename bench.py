@@ -55,6 +55,25 @@ def _peaks():
     return 6650.0, "fallback (earlier measurement on this pool)"
 
 
+def _tensor_peak():
+    """Sustained dense bf16 TFLOP/s (the figure for a kernel timed inside a long step)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"])
+    return 1400.0
+
+
+def _pass_roofline(shape, rows, ms):
+    """A pass against the larger of its two floors: streaming the weights once (HBM) and 2 x params x
+    rows flops on the tensor cores.  Past about 210 rows the second is the larger."""
+    peak, _ = _peaks()
+    t_hbm = shape.streamed_params * 2 / (peak * 1e9) * 1e3
+    t_tc = 2.0 * shape.streamed_params * rows / (_tensor_peak() * 1e12) * 1e3
+    return {"floor_hbm_ms": t_hbm, "floor_tensor_ms": t_tc, "bound": "hbm" if t_hbm >= t_tc else "tensor",
+            "frac_of_floor": max(t_hbm, t_tc) / ms}
+
+
 def _expected_tokens_per_step(tmpl, fraction):
     has_child = [False] * tmpl.N
     for p in tmpl.parent:
@@ -561,14 +580,14 @@ def run_attn_sweep():
 
 def _time_steps(ctx, steps, warm=4):
     for _ in range(warm):
-        ctx.step_enqueue(None)
+        ctx.step_batch_enqueue(None)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
-        ctx.step_enqueue(None)
+        ctx.step_batch_enqueue(None)
     e1.record()
     torch.cuda.synchronize()
-    ctx.step_finish()
+    ctx.step_batch_finish()
     return e0.elapsed_time(e1) / steps
 
 
@@ -582,7 +601,9 @@ def run_next_rows(args, shape):
       per node as the paper attaches them, plus the configuration's product-rule tree - next to
       the library in autoregressive mode.  The acceptance side comes from the stated synthetic model
       in synth/acceptance.py (no tuned model or dataset exists here): tokens per pass by seeded
-      simulation, tokens/s = tokens per pass / measured latency, speedup = tokens/s over AR tokens/s.
+      simulation, tokens/s = tokens per pass / measured latency, speedup = tokens/s over AR tokens/s;
+    * several sequences in one pass (a context of batch > 1): latency of the pass and aggregate
+      tokens/s for 1..5 sequences of the configuration's 69-row block, prompts of different lengths.
     """
     from paper_2401_12522_b200 import Bita, BitaError
     from paper_2401_12522_b200.build import build
@@ -648,8 +669,29 @@ def run_next_rows(args, shape):
         ms = _time_steps(ctx, steps)
         ctx.close()
         line.update(ms_per_step=ms, tokens_per_s=acc / ms * 1e3, speedup_vs_autoregressive=(acc / ms) / (1.0 / ar_ms),
-                    weights_hbm_frac=shape.streamed_params * 2 / ms / 1e6 / peak)
+                    weights_hbm_frac=shape.streamed_params * 2 / ms / 1e6 / peak, roofline=_pass_roofline(shape, rows, ms))
         print(json.dumps(line))
+    # ---- several sequences in one pass: each with its own prompt length, cache, tree and accepted length
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    rows = 1 + tmpl.N + tmpl.G * shape.n_mask
+    depth = max(tmpl.depths(), default=0)
+    acc = synth.tokens_per_pass(tmpl, shape.n_mask, model)["tokens_per_pass"]
+    B = 1
+    while B * rows <= 352 and B <= 16:
+        lens = [max(16, shape.prompt_len - 37 * b) for b in range(B)]
+        ctx = Bita(shape, weights, tmpl, C_max=shape.prompt_len + (steps + 8) * (depth + 1) + rows + 64, device=dev,
+                   batch=B)
+        for b in range(B):
+            ctx.prefill(prompt[:lens[b]], seq=b)
+        ms = _time_steps(ctx, steps)
+        ctx.close()
+        flops = 2.0 * shape.streamed_params * B * rows
+        print(json.dumps({"metric": "step_latency_by_batch", "workload": shape.name, "sequences": B, "rows": B * rows,
+                          "prompt_lens": lens, "ms_per_step": ms, "tokens_per_pass_model": acc * B,
+                          "tokens_per_s": acc * B / ms * 1e3, "speedup_vs_autoregressive": (acc * B / ms) / (1.0 / ar_ms),
+                          "weights_hbm_frac": shape.streamed_params * 2 / ms / 1e6 / peak,
+                          "tflops": flops / ms / 1e9, "roofline": _pass_roofline(shape, B * rows, ms)}))
+        B += 1
 
 
 def _spawn_ranks(n: int):

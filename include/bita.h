@@ -45,6 +45,7 @@ extern "C" {
 #define BITA_MAX_DEPTH 16
 #define BITA_MAX_TOPK 16            /* largest rank + 1 a template may use                            */
 #define BITA_MAX_MASK 8             /* mask tokens per group                                          */
+#define BITA_MAX_BATCH 16           /* sequences of one context; batch * rows per sequence <= BITA_MAX_ROWS */
 
 /* Model dimensions (the paper only says "LLaMA-2", Sec. 4.1): RMSNorm, rotary
  * embedding with half-split pairing, SwiGLU, no biases, untied LM head. */
@@ -95,7 +96,8 @@ typedef struct {
   const int32_t* attach;            /* G entries, -1 <= attach[g] < N, all distinct             */
 } bita_tree_template;
 
-/* KV cache: DEVICE, bf16, layout [L][H_kv][C_max][D] for keys and for values. */
+/* KV cache: DEVICE, bf16, layout [L][B][H_kv][C_max][D] for keys and for values, B = sequences
+ * of the context (1 for bita_init: [L][H_kv][C_max][D]). */
 typedef struct {
   void* k;
   void* v;
@@ -143,7 +145,35 @@ int bita_step(bita_ctx* ctx, bita_kv* kv, const int32_t* tree_tokens, bita_step_
 int bita_step_enqueue(bita_ctx* ctx, bita_kv* kv, const int32_t* tree_tokens_dev);
 int bita_step_finish(bita_ctx* ctx, bita_step_out* out);
 
-/* Back to the state after bita_init: empty cache, no last token, no tree. */
+/* ---- several sequences in one pass ----
+ * The paper measures one sequence at a time (Sec. 4.1, batch size 1); a weight-streaming pass costs
+ * nearly the same for a few hundred rows as for 69, so the same pass can carry the blocks of
+ * `batch` independent sequences: batch * (1 + N + G * n_mask) <= BITA_MAX_ROWS rows, sequence-major.
+ * Each sequence has its own cache slab, length, last token, drafted tree, verification walk
+ * (Algorithm 1, else-branch, once per sequence), accepted length and compaction; the sequences
+ * share the tree template and the weights only.  bita_init_batch(.., batch = 1, ..) is bita_init.
+ *   bita_prefill_seq        first pass of ONE sequence (0 <= seq < batch), as bita_prefill
+ *   bita_step_batch         tree_tokens: HOST [batch][N] or NULL; out: HOST array of `batch` records
+ *   bita_step_batch_enqueue tree_tokens_dev: DEVICE [batch][N] or NULL; only enqueues
+ *   bita_step_batch_finish  waits, fills `batch` records; BITA_ERR_NOT_PREFILLED unless every sequence was prefilled
+ *   bita_rewind_seq         bita_rewind for one sequence
+ * bita_step / bita_step_enqueue / bita_step_finish / bita_prefill / bita_rewind act on sequence 0 and
+ * return BITA_ERR_INVALID_ARG on a context of more than one sequence (the step calls). */
+int bita_workspace_bytes_batch(const bita_model_dims* dims, const bita_tree_template* tmpl, int n_mask,
+                               int32_t batch, size_t* out_bytes);
+int bita_init_batch(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w,
+                    const bita_tree_template* tmpl, int n_mask, int32_t batch, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+int bita_prefill_seq(bita_ctx* ctx, bita_kv* kv, int32_t seq, const int32_t* tokens, int32_t count,
+                     bita_step_out* out);
+int bita_step_batch(bita_ctx* ctx, bita_kv* kv, const int32_t* tree_tokens, bita_step_out* out);
+int bita_step_batch_enqueue(bita_ctx* ctx, bita_kv* kv, const int32_t* tree_tokens_dev);
+int bita_step_batch_finish(bita_ctx* ctx, bita_step_out* out);
+int bita_rewind_seq(bita_ctx* ctx, bita_kv* kv, int32_t seq, int32_t new_len, int32_t last_token);
+/* Sequences of the context. */
+int bita_batch(const bita_ctx* ctx);
+
+/* Back to the state after bita_init: empty caches, no last tokens, no trees (all sequences). */
 int bita_reset(bita_ctx* ctx, bita_kv* kv);
 
 /* Cut the decoding state back (Algorithm 1 cuts the output at <EOS>; a caller that goes on after
@@ -196,7 +226,7 @@ int bita_probe_wait_timeout(bita_ctx* ctx, uint64_t limit_ns);
 int bita_set_kernel_timing(bita_ctx* ctx, int on);
 int bita_get_kernel_timing(bita_ctx* ctx, float* ms, int32_t* launches);
 
-/* Rows of the packed block of bita_step for this context (1 + N + G * n_mask). */
+/* Rows one sequence contributes to the packed block of a step (1 + N + G * n_mask). */
 int bita_block_rows(const bita_ctx* ctx);
 /* Number of kernel launches the most recent bita_step / bita_step_enqueue / bita_prefill made. */
 int bita_last_launch_count(const bita_ctx* ctx);

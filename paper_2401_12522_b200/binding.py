@@ -10,7 +10,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libbita.so")
 
-MAX_NODES, MAX_ROWS, MAX_DEPTH, MAX_TOPK, MAX_MASK = 160, 352, 16, 16, 8
+MAX_NODES, MAX_ROWS, MAX_DEPTH, MAX_TOPK, MAX_MASK, MAX_BATCH = 160, 352, 16, 16, 8, 16
 
 
 class BitaError(RuntimeError):
@@ -53,6 +53,15 @@ def _signatures():
         "bita_workspace_bytes": [C.POINTER(ModelDims), C.POINTER(TreeTemplate), C.c_int, C.POINTER(sz)],
         "bita_init": [C.POINTER(vp), C.POINTER(ModelDims), C.POINTER(Weights), C.POINTER(TreeTemplate), C.c_int,
                       vp, sz, vp],
+        "bita_workspace_bytes_batch": [C.POINTER(ModelDims), C.POINTER(TreeTemplate), C.c_int, i32, C.POINTER(sz)],
+        "bita_init_batch": [C.POINTER(vp), C.POINTER(ModelDims), C.POINTER(Weights), C.POINTER(TreeTemplate), C.c_int,
+                            i32, vp, sz, vp],
+        "bita_prefill_seq": [vp, C.POINTER(KV), i32, C.POINTER(i32), i32, C.POINTER(StepOut)],
+        "bita_step_batch": [vp, C.POINTER(KV), C.POINTER(i32), C.POINTER(StepOut)],
+        "bita_step_batch_enqueue": [vp, C.POINTER(KV), vp],
+        "bita_step_batch_finish": [vp, C.POINTER(StepOut)],
+        "bita_rewind_seq": [vp, C.POINTER(KV), i32, i32, i32],
+        "bita_batch": [vp],
         "bita_prefill": [vp, C.POINTER(KV), C.POINTER(i32), i32, C.POINTER(StepOut)],
         "bita_step": [vp, C.POINTER(KV), C.POINTER(i32), C.POINTER(StepOut)],
         "bita_step_enqueue": [vp, C.POINTER(KV), vp],
@@ -118,8 +127,9 @@ def _i32_array(vals: Sequence[int]):
 class Bita:
     """One decoding context: owns (through torch) the workspace and the KV cache it hands to the library."""
 
-    def __init__(self, shape, weights: Dict, template, *, C_max: int, stream=None, device="cuda:0"):
+    def __init__(self, shape, weights: Dict, template, *, C_max: int, stream=None, device="cuda:0", batch: int = 1):
         self.device = torch.device(device)
+        self.batch = batch
         self.stream = stream
         self.shape = shape
         self.template = template
@@ -145,21 +155,23 @@ class Bita:
             setattr(w, k, C.cast(arr, C.POINTER(C.c_void_p)))
         self._w = w
         need = C.c_size_t(0)
-        _check(lib.bita_workspace_bytes(C.byref(self.dims), C.byref(self.tmpl), self.n_mask, C.byref(need)),
-               "bita_workspace_bytes")
+        _check(lib.bita_workspace_bytes_batch(C.byref(self.dims), C.byref(self.tmpl), self.n_mask, batch,
+                                              C.byref(need)), "bita_workspace_bytes_batch")
         self.workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
         ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
-        kv_shape = (L, shape.H_kv, C_max, shape.D)
+        # [L][B][H_kv][C_max][D]; with one sequence the B axis is left out
+        kv_shape = (L, shape.H_kv, C_max, shape.D) if batch == 1 else (L, batch, shape.H_kv, C_max, shape.D)
         self.k_cache = torch.zeros(kv_shape, dtype=torch.bfloat16, device=self.device)
         self.v_cache = torch.zeros(kv_shape, dtype=torch.bfloat16, device=self.device)
         self.kv = KV(self.k_cache.data_ptr(), self.v_cache.data_ptr(), C_max)
         self._ctx = C.c_void_p(0)
         torch.cuda.synchronize(self.device)
-        _check(lib.bita_init(C.byref(self._ctx), C.byref(self.dims), C.byref(w), C.byref(self.tmpl), self.n_mask,
-                             C.c_void_p(ws_ptr), need.value, _stream_handle(stream)), "bita_init")
+        _check(lib.bita_init_batch(C.byref(self._ctx), C.byref(self.dims), C.byref(w), C.byref(self.tmpl), self.n_mask,
+                                   batch, C.c_void_p(ws_ptr), need.value, _stream_handle(stream)), "bita_init_batch")
         self.rows = lib.bita_block_rows(self._ctx)
         self._debug = None
         self._out = StepOut()
+        self._outs = (StepOut * batch)()
 
     @staticmethod
     def _all_tensors(weights):
@@ -172,10 +184,27 @@ class Bita:
                 yield k, v
 
     # ---- the three calls -------------------------------------------------------------------
-    def prefill(self, tokens: Sequence[int]) -> Dict:
+    def prefill(self, tokens: Sequence[int], seq: int = 0) -> Dict:
         arr = _i32_array(tokens)
-        _check(lib.bita_prefill(self._ctx, C.byref(self.kv), arr, len(tokens), C.byref(self._out)), "bita_prefill")
+        _check(lib.bita_prefill_seq(self._ctx, C.byref(self.kv), seq, arr, len(tokens), C.byref(self._out)),
+               "bita_prefill_seq")
         return self._record()
+
+    # ---- several sequences in one pass ------------------------------------------------------
+    def step_batch(self, tree_tokens: Optional[Sequence[Sequence[int]]] = None):
+        """One pass over all sequences; `tree_tokens` = one token list per sequence, or None."""
+        arr = None if tree_tokens is None else _i32_array([t for seq in tree_tokens for t in seq])
+        _check(lib.bita_step_batch(self._ctx, C.byref(self.kv), arr, self._outs), "bita_step_batch")
+        return [self._record(self._outs[b]) for b in range(self.batch)]
+
+    def step_batch_enqueue(self, tree_tokens_dev: Optional[torch.Tensor] = None):
+        if tree_tokens_dev is not None:
+            assert tree_tokens_dev.dtype == torch.int32 and tree_tokens_dev.is_cuda and tree_tokens_dev.is_contiguous()
+        _check(lib.bita_step_batch_enqueue(self._ctx, C.byref(self.kv), _ptr(tree_tokens_dev)), "bita_step_batch_enqueue")
+
+    def step_batch_finish(self):
+        _check(lib.bita_step_batch_finish(self._ctx, self._outs), "bita_step_batch_finish")
+        return [self._record(self._outs[b]) for b in range(self.batch)]
 
     def step(self, tree_tokens: Optional[Sequence[int]] = None) -> Dict:
         arr = None if tree_tokens is None else _i32_array(tree_tokens)
@@ -194,12 +223,12 @@ class Bita:
     def reset(self):
         _check(lib.bita_reset(self._ctx, C.byref(self.kv)), "bita_reset")
 
-    def rewind(self, new_len: int, last_token: int):
-        _check(lib.bita_rewind(self._ctx, C.byref(self.kv), new_len, last_token), "bita_rewind")
+    def rewind(self, new_len: int, last_token: int, seq: int = 0):
+        _check(lib.bita_rewind_seq(self._ctx, C.byref(self.kv), seq, new_len, last_token), "bita_rewind_seq")
 
     # ---- helpers ---------------------------------------------------------------------------
-    def _record(self) -> Dict:
-        o = self._out
+    def _record(self, o=None) -> Dict:
+        o = self._out if o is None else o
         n = o.n_out
         return dict(status=o.status, n_out=n, new_len=o.new_len, out_tokens=list(o.out_tokens[:n]),
                     accepted_idx=list(o.accepted_idx[:max(0, n - 1)]), next_tree=list(o.next_tree[:self.template.N]))

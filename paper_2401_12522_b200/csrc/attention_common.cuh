@@ -22,7 +22,8 @@ struct AttnArgs {
   const bf16* prompt_k;      // [H_kv][P][D] or null
   const bf16* prompt_v;
   const uint8_t* sees_prompt;  // [B][M] or null
-  const int32_t* ctx_len;    // [B]
+  const int32_t* ctx_len;    // C of sequence b at ctx_len[b * ctx_len_stride]
+  int32_t ctx_len_stride;
   int32_t vis_batch_stride;  // words between sequences (0 = shared)
   int32_t sp_batch_stride;
   bf16* out;                 // [B][M][H*D]

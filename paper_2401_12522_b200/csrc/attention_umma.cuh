@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1) k_attn_umma(const __grid_consta
   if (threadIdx.x == 0) pdl_launch();
 
   // ---- key chunks of this slice (the context length was settled by an earlier pass)
-  const int C = a.ctx_len[b];
+  const int C = a.ctx_len[(size_t)b * a.ctx_len_stride];
   const int n_cache = C + a.M;
   const int cache_chunks = (n_cache + AU_KEYS - 1) / AU_KEYS;
   const bool has_prompt = a.P > 0 && a.prompt_k && a.prompt_v && a.sees_prompt;

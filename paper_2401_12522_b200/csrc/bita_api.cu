@@ -67,6 +67,7 @@ inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 // Host description of a packed block; `upload_plan` writes it into a device region and fills `dev`.
 struct HostPlan {
   int M = 0, W = 0, N = 0, G = 0, n_mask = 0, k_max = 1, n_query = 0, max_depth = 0;
+  int B = 1, seq0 = 0;     // sequences in the block (M = rows of one of them), first sequence
   std::vector<int32_t> row_kind, row_idx, rel_pos, parent, rank, depth, group_of;
   std::vector<uint8_t> sees_prompt;
   std::vector<uint32_t> vis;
@@ -77,16 +78,20 @@ constexpr size_t PLAN_REGION_BYTES =
     sizeof(int32_t) * (3 * BITA_MAX_ROWS + BITA_MAX_ROWS * (BITA_MAX_ROWS / 32) + 3 * BITA_MAX_NODES +
                        (BITA_MAX_NODES + 1)) + BITA_MAX_ROWS + 1024;
 
-// Step block (Sec. 3.2, Appendix B): root, tree nodes, G groups of n mask tokens.
-int build_step_plan(const bita_tree_template* t, int n_mask, HostPlan* p) {
+// Step block (Sec. 3.2, Appendix B): root, tree nodes, G groups of n mask tokens, for each of
+// `batch` sequences (the tables describe one sequence; the block repeats them sequence-major).
+int build_step_plan(const bita_tree_template* t, int n_mask, int batch, HostPlan* p) {
+  if (batch < 1 || batch > BITA_MAX_BATCH) return BITA_ERR_INVALID_ARG;
   if (!t || t->N < 0 || t->N > BITA_MAX_NODES || t->G < 0) return BITA_ERR_BAD_TEMPLATE;
   if (t->N > 0 && (!t->parent || !t->rank)) return BITA_ERR_BAD_TEMPLATE;
   if (t->G > 0 && !t->attach) return BITA_ERR_BAD_TEMPLATE;
   if (n_mask < 0 || n_mask > BITA_MAX_MASK) return BITA_ERR_INVALID_ARG;
   const int N = t->N, G = t->G;
   const long rows = 1L + N + (long)G * n_mask;
-  if (rows > BITA_MAX_ROWS) return BITA_ERR_BAD_TEMPLATE;
+  if (rows * batch > BITA_MAX_ROWS) return BITA_ERR_BAD_TEMPLATE;
   p->M = (int)rows;
+  p->B = batch;
+  p->seq0 = 0;
   p->W = (p->M + 31) / 32;
   p->N = N;
   p->G = G;
@@ -147,9 +152,11 @@ int build_step_plan(const bita_tree_template* t, int n_mask, HostPlan* p) {
 
 // Prefill chunk (Algorithm 1, t = 1): `cnt` query tokens, causal; the last chunk is followed by
 // one group of n_mask mask tokens attached to the final query token.
-void build_prefill_plan(int cnt, int n_mask, bool last, int k_max, HostPlan* p) {
+void build_prefill_plan(int cnt, int n_mask, bool last, int k_max, int seq, HostPlan* p) {
   const int M = cnt + (last ? n_mask : 0);
   p->M = M;
+  p->B = 1;
+  p->seq0 = seq;
   p->W = (M + 31) / 32;
   p->N = 0;
   p->G = last ? 1 : 0;
@@ -191,7 +198,7 @@ int upload_plan(HostPlan* p, void* region, cudaStream_t stream) {
     return (const uint8_t*)region + at;
   };
   DevPlan& d = p->dev;
-  d.M = p->M; d.W = p->W; d.N = p->N; d.G = p->G; d.n_mask = p->n_mask; d.k_max = p->k_max;
+  d.M = p->M; d.B = p->B; d.seq0 = p->seq0; d.W = p->W; d.N = p->N; d.G = p->G; d.n_mask = p->n_mask; d.k_max = p->k_max;
   d.n_query = p->n_query; d.max_depth = p->max_depth;
   d.row_kind = (const int32_t*)put(p->row_kind.data(), p->row_kind.size() * 4);
   d.row_idx = (const int32_t*)put(p->row_idx.data(), p->row_idx.size() * 4);
@@ -371,6 +378,7 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   if (!p.wait_ns) p.wait_ns = TC_WAIT_LIMIT_NS;
   int splits = effective_splits(g, n_pad);
   p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.dual = g.dual;
+  if (p.rows_per_seq < 1) p.rows_per_seq = M;
   int cols = 32;
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
@@ -454,12 +462,12 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   t.gemm_cnt = (int32_t*)take((size_t)GEMM_KINDS * TC_MAX_TILES * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
-  t.state = (DevState*)take(sizeof(DevState));
-  t.rec = (DevRecord*)take(sizeof(DevRecord));
+  t.state = (DevState*)take(sizeof(DevState) * BITA_MAX_BATCH);      // one per sequence
+  t.rec = (DevRecord*)take(sizeof(DevRecord) * BITA_MAX_BATCH);
   t.plan_step = take(PLAN_REGION_BYTES);
   t.plan_prefill = take(PLAN_REGION_BYTES);
   t.query_tokens = (int32_t*)take(PREFILL_CHUNK * 4);
-  t.tree_in = (int32_t*)take(BITA_MAX_NODES * 4);
+  t.tree_in = (int32_t*)take((size_t)BITA_MAX_ROWS * 4);               // [B][N] tree tokens of a step, B * N < rows
   if (b) *b = t;
   return off;
 }
@@ -474,9 +482,10 @@ struct bita_ctx {
   cudaStream_t stream;
   Buffers b;
   HostPlan step_plan, prefill_plan;
-  DevRecord* rec_host;      // pinned
-  int len_upper;            // upper bound of the device-side cache length
-  bool prefilled;
+  int B;                    // sequences decoded together (1 for bita_init)
+  DevRecord* rec_host;      // pinned, one record per sequence
+  std::vector<int> len_upper;       // per sequence: upper bound of the device-side cache length
+  std::vector<char> prefilled;      // per sequence
   float* dbg;
   int launches;
   std::vector<GemmDesc> d_qkv, d_o, d_gu, d_dn;
@@ -634,14 +643,17 @@ int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std:
 int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_dev, bool want_logits) {
   const bita_model_dims& m = c->m;
   const DevPlan& P = hp.dev;
-  const int M = P.M;
+  const int M = P.M * P.B;                                   // rows of the block: P.B sequences of P.M rows
   cudaStream_t s = c->stream;
   Buffers& b = c->b;
   c->ev_family.clear();
   c->ev_count.clear();
   c->last_rows = M;
   mark(c, 2);
-  const size_t layer_kv = (size_t)m.H_kv * kv->C_max * m.D;
+  const size_t seq_kv = (size_t)m.H_kv * kv->C_max * m.D;      // one sequence's slab of a layer
+  const size_t layer_kv = seq_kv * c->B;                       // cache layout [L][B][H_kv][C_max][D]
+  const size_t block_kv = seq_kv * P.seq0;                     // the block's first sequence within a layer
+  const DevState* st0 = b.state + P.seq0;
   const bool pdl = c->pdl;
   int rc;
   const int n_slots = 2 * m.L + 1;
@@ -666,8 +678,10 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
   struct ProjOp { const GemmDesc* g; const bf16* X; GemmTcParams p; };
   auto op_qkv = [&](int l) {
     GemmTcParams p{};
-    p.mode = EPI_QKV; p.q = b.q; p.kc = (bf16*)kv->k + (size_t)l * layer_kv; p.vc = (bf16*)kv->v + (size_t)l * layer_kv;
-    p.rope_blk = b.rope_blk; p.len_ptr = &b.state->len; p.H = m.H; p.H_kv = m.H_kv; p.D = m.D; p.C_max = kv->C_max;
+    p.mode = EPI_QKV; p.q = b.q;
+    p.kc = (bf16*)kv->k + (size_t)l * layer_kv + block_kv; p.vc = (bf16*)kv->v + (size_t)l * layer_kv + block_kv;
+    p.rope_blk = b.rope_blk; p.len_ptr = &st0->len; p.len_stride = (int32_t)(sizeof(DevState) / 4);
+    p.seq_stride = (long long)seq_kv; p.H = m.H; p.H_kv = m.H_kv; p.D = m.D; p.C_max = kv->C_max;
     return ProjOp{&c->d_qkv[l], b.xn, with_norm(p, 2 * l)};       // attention RMSNorm scale + q/k/v + RoPE + cache write
   };
   auto op_o = [&](int l) {   // output projection + residual add; leaves x * g_ffn and the row statistics
@@ -682,16 +696,17 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     const void* g_next = l + 1 < m.L ? c->g_attn[l + 1] : c->g_final;
     return ProjOp{&c->d_dn[l], b.hf, epi_resid(g_next, 2 * l + 2)};
   };
-  auto single = [&](const ProjOp& o) { return gemm(c, *o.g, o.X, M, o.p); };
+  auto single = [&](ProjOp o) { o.p.rows_per_seq = P.M; return gemm(c, *o.g, o.X, M, o.p); };
   for (int l = 0; l < m.L; ++l) {
-    bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv;
-    bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv;
+    bf16* kc = (bf16*)kv->k + (size_t)l * layer_kv + block_kv;
+    bf16* vc = (bf16*)kv->v + (size_t)l * layer_kv + block_kv;
     if ((rc = single(op_qkv(l)))) return rc;
     AttnArgs a{};
     a.q = b.q; a.k = kc; a.v = vc; a.vis = P.vis; a.prompt_k = (const bf16*)c->prompt_k[l];
-    a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &b.state->len;
+    a.prompt_v = (const bf16*)c->prompt_v[l]; a.sees_prompt = P.sees_prompt; a.ctx_len = &st0->len;
+    a.ctx_len_stride = (int32_t)(sizeof(DevState) / 4);
     a.vis_batch_stride = 0; a.sp_batch_stride = 0; a.out = b.att; a.part_ml = b.part_ml; a.part_acc = b.part_acc;
-    a.B = 1; a.M = M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
+    a.B = P.B; a.M = P.M; a.W = P.W; a.H = m.H; a.H_kv = m.H_kv; a.D = m.D; a.P = m.P; a.C_max = kv->C_max;
     a.status = &b.state->status;
     a.wait_ns = c->wait_ns;
     {
@@ -717,6 +732,7 @@ int run_block(bita_ctx* c, bita_kv* kv, const HostPlan& hp, const int32_t* tree_
     hp.cand = b.cand;
     hp.row_kind = P.row_kind;
     hp.k_max = P.k_max;
+    hp.rows_per_seq = P.M;
     if ((rc = gemm(c, c->d_head, b.xn, M, with_norm(hp, 2 * m.L)))) return rc;
     mark(c, 2);
     if ((rc = launch(s, pdl, dim3(M), dim3(256), 0, 1, k_select_merge, P, (const unsigned long long*)b.cand,
@@ -742,19 +758,24 @@ void fill_out(const DevRecord* r, bita_step_out* out) {
 
 extern "C" {
 
-int bita_workspace_bytes(const bita_model_dims* dims, const bita_tree_template* tmpl, int n_mask, size_t* out_bytes) {
+int bita_workspace_bytes_batch(const bita_model_dims* dims, const bita_tree_template* tmpl, int n_mask, int32_t batch,
+                               size_t* out_bytes) {
   if (!out_bytes) return BITA_ERR_INVALID_ARG;
   int rc = check_dims(dims);
   if (rc) return rc;
   HostPlan p;
-  rc = build_step_plan(tmpl, n_mask, &p);
+  rc = build_step_plan(tmpl, n_mask, batch, &p);
   if (rc) return rc;
   *out_bytes = carve(*dims, nullptr, nullptr);
   return BITA_OK;
 }
 
-int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w, const bita_tree_template* tmpl,
-              int n_mask, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+int bita_workspace_bytes(const bita_model_dims* dims, const bita_tree_template* tmpl, int n_mask, size_t* out_bytes) {
+  return bita_workspace_bytes_batch(dims, tmpl, n_mask, 1, out_bytes);
+}
+
+int bita_init_batch(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w, const bita_tree_template* tmpl,
+                    int n_mask, int32_t batch, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!out || !w || !workspace) return BITA_ERR_INVALID_ARG;
   *out = nullptr;
   int rc = check_dims(dims);
@@ -766,7 +787,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   if (dims->P > 0 && (!w->prompt_k || !w->prompt_v)) return BITA_ERR_INVALID_ARG;
   bita_ctx* c = new (std::nothrow) bita_ctx();
   if (!c) return BITA_ERR_INVALID_ARG;
-  rc = build_step_plan(tmpl, n_mask, &c->step_plan);
+  rc = build_step_plan(tmpl, n_mask, batch, &c->step_plan);
   if (rc) { delete c; return rc; }
   if (((uintptr_t)workspace % ALIGN) || workspace_bytes < carve(*dims, nullptr, nullptr)) {
     delete c;
@@ -774,6 +795,7 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   }
   c->m = *dims;
   c->n_mask = n_mask;
+  c->B = batch;
   c->stream = (cudaStream_t)cuda_stream;
   c->tok_emb = w->tok_emb; c->mask_emb = w->mask_emb; c->g_final = w->g_final; c->lm_head = w->lm_head;
   const int L = dims->L;
@@ -796,11 +818,11 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   c->wait_ns = TC_WAIT_LIMIT_NS;
   c->last_rows = 0;
 
-  c->prefilled = false;
-  c->len_upper = 0;
+  c->prefilled.assign(batch, 0);
+  c->len_upper.assign(batch, 0);
   auto fail = [&](int code) { if (c->rec_host) cudaFreeHost(c->rec_host); delete c; return code; };
-  if (cudaMallocHost((void**)&c->rec_host, sizeof(DevRecord)) != cudaSuccess) return fail(BITA_ERR_CUDA);
-  memset(c->rec_host, 0, sizeof(DevRecord));
+  if (cudaMallocHost((void**)&c->rec_host, sizeof(DevRecord) * BITA_MAX_BATCH) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  memset(c->rec_host, 0, sizeof(DevRecord) * BITA_MAX_BATCH);
   // rotary table in double precision: angle = pos * theta^(-2j/D)
   {
     const int half = dims->D / 2, npos = dims->C_max + 64;
@@ -834,47 +856,58 @@ int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w
   if (rc) return fail(rc);
   if (cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
-  k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
+  k_reset_state<<<BITA_MAX_BATCH, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
   return BITA_OK;
 }
+
+int bita_init(bita_ctx** out, const bita_model_dims* dims, const bita_weights* w, const bita_tree_template* tmpl,
+              int n_mask, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return bita_init_batch(out, dims, w, tmpl, n_mask, 1, workspace, workspace_bytes, cuda_stream);
+}
+
+int bita_batch(const bita_ctx* c) { return c ? c->B : BITA_ERR_INVALID_ARG; }
 
 int bita_reset(bita_ctx* c, bita_kv* kv) {
   if (!c || !kv) return BITA_ERR_INVALID_ARG;
   // a pass that gave up on a wait may have left split counters half way
   CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream));
   for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
-  k_reset_state<<<1, 128, 0, c->stream>>>(c->b.state);
+  k_reset_state<<<BITA_MAX_BATCH, 128, 0, c->stream>>>(c->b.state);
   CU_TRY(cudaStreamSynchronize(c->stream));
-  c->prefilled = false;
-  c->len_upper = 0;
+  c->prefilled.assign(c->B, 0);
+  c->len_upper.assign(c->B, 0);
+  return BITA_OK;
+}
+
+int bita_rewind_seq(bita_ctx* c, bita_kv* kv, int32_t seq, int32_t new_len, int32_t last_token) {
+  if (!c || !kv || seq < 0 || seq >= c->B) return BITA_ERR_INVALID_ARG;
+  if (!c->prefilled[seq]) return BITA_ERR_NOT_PREFILLED;
+  if (new_len < 0 || new_len > c->len_upper[seq] || last_token < 0 || last_token >= c->m.V) return BITA_ERR_INVALID_ARG;
+  k_set_state<<<1, 128, 0, c->stream>>>(c->b.state + seq, new_len, last_token);
+  CU_TRY(cudaGetLastError());
+  c->len_upper[seq] = new_len;
   return BITA_OK;
 }
 
 int bita_rewind(bita_ctx* c, bita_kv* kv, int32_t new_len, int32_t last_token) {
-  if (!c || !kv) return BITA_ERR_INVALID_ARG;
-  if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
-  if (new_len < 0 || new_len > c->len_upper || last_token < 0 || last_token >= c->m.V) return BITA_ERR_INVALID_ARG;
-  k_set_state<<<1, 128, 0, c->stream>>>(c->b.state, new_len, last_token);
-  CU_TRY(cudaGetLastError());
-  c->len_upper = new_len;
-  return BITA_OK;
+  return bita_rewind_seq(c, kv, 0, new_len, last_token);
 }
 
-int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count, bita_step_out* out) {
-  if (!c || !kv || !kv->k || !kv->v || !tokens || count < 1) return BITA_ERR_INVALID_ARG;
+int bita_prefill_seq(bita_ctx* c, bita_kv* kv, int32_t seq, const int32_t* tokens, int32_t count, bita_step_out* out) {
+  if (!c || !kv || !kv->k || !kv->v || !tokens || count < 1 || seq < 0 || seq >= c->B) return BITA_ERR_INVALID_ARG;
   if (kv->C_max != c->m.C_max) return BITA_ERR_INVALID_ARG;
   for (int i = 0; i < count; ++i)
     if (tokens[i] < 0 || tokens[i] >= c->m.V) return BITA_ERR_INVALID_ARG;
-  if ((long)c->len_upper + count + c->n_mask > kv->C_max) return BITA_ERR_KV_FULL;
+  if ((long)c->len_upper[seq] + count + c->n_mask > kv->C_max) return BITA_ERR_KV_FULL;
   c->launches = 0;
   // Equal blocks, as few as the row limit allows: every block streams all the weights once.
   int blocks_left = (count + PREFILL_CHUNK - 1) / PREFILL_CHUNK;
   for (int done = 0; done < count; --blocks_left) {
     const int cnt = (count - done + blocks_left - 1) / blocks_left;
     const bool last = done + cnt == count;
-    build_prefill_plan(cnt, c->n_mask, last, c->step_plan.k_max, &c->prefill_plan);
+    build_prefill_plan(cnt, c->n_mask, last, c->step_plan.k_max, seq, &c->prefill_plan);
     int rc = upload_plan(&c->prefill_plan, c->b.plan_prefill, c->stream);
     if (rc) return rc;
     CU_TRY(cudaMemcpyAsync(c->b.query_tokens, tokens + done, cnt * 4, cudaMemcpyHostToDevice, c->stream));
@@ -887,56 +920,83 @@ int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count,
     CU_TRY(cudaStreamSynchronize(c->stream));   // the plan region and token buffer are reused by the next chunk
     done += cnt;
   }
-  CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
+  DevRecord* rh = c->rec_host + seq;
+  CU_TRY(cudaMemcpyAsync(rh, c->b.rec + seq, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
   CU_TRY(cudaStreamSynchronize(c->stream));
-  c->len_upper = c->rec_host->new_len;
-  c->prefilled = true;
-  if (out) fill_out(c->rec_host, out);
-  return c->rec_host->status ? BITA_ERR_TIMEOUT : BITA_OK;
+  c->len_upper[seq] = rh->new_len;
+  c->prefilled[seq] = 1;
+  if (out) fill_out(rh, out);
+  return rh->status ? BITA_ERR_TIMEOUT : BITA_OK;
 }
 
-int bita_step_enqueue(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens_dev) {
+int bita_prefill(bita_ctx* c, bita_kv* kv, const int32_t* tokens, int32_t count, bita_step_out* out) {
+  return bita_prefill_seq(c, kv, 0, tokens, count, out);
+}
+
+int bita_step_batch_enqueue(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens_dev) {
   if (!c || !kv || !kv->k || !kv->v) return BITA_ERR_INVALID_ARG;
   if (kv->C_max != c->m.C_max) return BITA_ERR_INVALID_ARG;
-  if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
-  if ((long)c->len_upper + c->step_plan.M > kv->C_max) return BITA_ERR_KV_FULL;
+  for (int b = 0; b < c->B; ++b) {
+    if (!c->prefilled[b]) return BITA_ERR_NOT_PREFILLED;
+    if ((long)c->len_upper[b] + c->step_plan.M > kv->C_max) return BITA_ERR_KV_FULL;
+  }
   c->launches = 0;
   int rc = run_block(c, kv, c->step_plan, tree_tokens_dev, true);
   if (rc) return rc;
-  if ((rc = launch(c->stream, c->pdl, dim3(1), dim3(32), 0, 1, k_accept, c->step_plan.dev, c->b.state,
+  if ((rc = launch(c->stream, c->pdl, dim3(c->B), dim3(32), 0, 1, k_accept, c->step_plan.dev, c->b.state,
                    (const int32_t*)c->b.row_token, (const int32_t*)c->b.sel_id, c->b.rec)))
     return rc;
-  if ((rc = launch(c->stream, c->pdl, dim3(c->m.L * c->m.H_kv), dim3(64), 0, 1, k_compact, (const DevRecord*)c->b.rec,
-                   c->m.D, kv->C_max, (bf16*)kv->k, (bf16*)kv->v)))
+  if ((rc = launch(c->stream, c->pdl, dim3(c->m.L * c->m.H_kv, c->B), dim3(64), 0, 1, k_compact,
+                   (const DevRecord*)c->b.rec, c->m.D, kv->C_max, c->m.H_kv, c->B, (bf16*)kv->k, (bf16*)kv->v)))
     return rc;
   c->launches += 2;
   CU_TRY(cudaGetLastError());
-  CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord), cudaMemcpyDeviceToHost, c->stream));
-  c->len_upper += c->step_plan.max_depth + 1;
+  CU_TRY(cudaMemcpyAsync(c->rec_host, c->b.rec, sizeof(DevRecord) * c->B, cudaMemcpyDeviceToHost, c->stream));
+  for (int b = 0; b < c->B; ++b) c->len_upper[b] += c->step_plan.max_depth + 1;
   return BITA_OK;
 }
 
-int bita_step_finish(bita_ctx* c, bita_step_out* out) {
+int bita_step_batch_finish(bita_ctx* c, bita_step_out* out) {
   if (!c || !out) return BITA_ERR_INVALID_ARG;
   CU_TRY(cudaStreamSynchronize(c->stream));
-  c->len_upper = c->rec_host->new_len;
-  fill_out(c->rec_host, out);
-  return c->rec_host->status ? BITA_ERR_TIMEOUT : BITA_OK;
+  int status = 0;
+  for (int b = 0; b < c->B; ++b) {
+    c->len_upper[b] = c->rec_host[b].new_len;
+    fill_out(c->rec_host + b, out + b);
+    if (c->rec_host[b].status) status = c->rec_host[b].status;
+  }
+  return status ? BITA_ERR_TIMEOUT : BITA_OK;
 }
 
-int bita_step(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens, bita_step_out* out) {
+int bita_step_batch(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens, bita_step_out* out) {
   if (!c || !out) return BITA_ERR_INVALID_ARG;
   const int32_t* dev = nullptr;
-  if (tree_tokens && c->step_plan.N > 0) {
-    for (int i = 0; i < c->step_plan.N; ++i)
+  const int n = c->B * c->step_plan.N;
+  if (tree_tokens && n > 0) {
+    for (int i = 0; i < n; ++i)
       if (tree_tokens[i] < -1 || tree_tokens[i] >= c->m.V) return BITA_ERR_INVALID_ARG;
-    if (!c->prefilled) return BITA_ERR_NOT_PREFILLED;
-    CU_TRY(cudaMemcpyAsync(c->b.tree_in, tree_tokens, c->step_plan.N * 4, cudaMemcpyHostToDevice, c->stream));
+    for (int b = 0; b < c->B; ++b)
+      if (!c->prefilled[b]) return BITA_ERR_NOT_PREFILLED;
+    CU_TRY(cudaMemcpyAsync(c->b.tree_in, tree_tokens, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
     dev = c->b.tree_in;
   }
-  int rc = bita_step_enqueue(c, kv, dev);
+  int rc = bita_step_batch_enqueue(c, kv, dev);
   if (rc) return rc;
-  return bita_step_finish(c, out);
+  return bita_step_batch_finish(c, out);
+}
+
+/* The batch-1 calls are the batch calls of a context with one sequence. */
+int bita_step_enqueue(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens_dev) {
+  if (c && c->B != 1) return BITA_ERR_INVALID_ARG;
+  return bita_step_batch_enqueue(c, kv, tree_tokens_dev);
+}
+int bita_step_finish(bita_ctx* c, bita_step_out* out) {
+  if (c && c->B != 1) return BITA_ERR_INVALID_ARG;
+  return bita_step_batch_finish(c, out);
+}
+int bita_step(bita_ctx* c, bita_kv* kv, const int32_t* tree_tokens, bita_step_out* out) {
+  if (c && c->B != 1) return BITA_ERR_INVALID_ARG;
+  return bita_step_batch(c, kv, tree_tokens, out);
 }
 
 int bita_set_debug_buffer(bita_ctx* c, void* dev_buf, size_t bytes) {
@@ -1098,7 +1158,7 @@ int tree_attention_impl(const void* q, const void* k, const void* v, const uint3
   const int W = (M + 31) / 32;
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
-  a.ctx_len = ctx_len; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
+  a.ctx_len = ctx_len; a.ctx_len_stride = 1; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
   // workspace: partial results of the key slices (used when the slices do not merge inside a cluster)
   a.part_ml = (float*)workspace;
   a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));

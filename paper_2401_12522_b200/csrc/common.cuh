@@ -18,9 +18,13 @@ typedef __nv_bfloat16 bf16;
 // Row kinds of a packed block.
 enum RowKind : int32_t { ROW_ROOT = 0, ROW_NODE = 1, ROW_MASK = 2, ROW_QUERY = 3 };
 
-// Layout of one packed block as the kernels see it (all pointers DEVICE).
+// Layout of one packed block as the kernels see it (all pointers DEVICE).  A block holds the rows
+// of B sequences, sequence-major: global row b * M + r is row r of the block's b-th sequence, which
+// is sequence seq0 + b of the context.  Every table below describes ONE sequence's M rows.
 struct DevPlan {
-  int32_t M;                  // rows
+  int32_t M;                  // rows per sequence
+  int32_t B;                  // sequences in the block
+  int32_t seq0;               // first of them
   int32_t W;                  // 32-bit words per visibility row = ceil(M / 32)
   int32_t N;                  // tree nodes
   int32_t G;                  // mask groups

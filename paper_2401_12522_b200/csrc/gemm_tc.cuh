@@ -82,6 +82,7 @@ __device__ __forceinline__ unsigned long long sumsq_to_fixed(float v) {
 
 struct GemmTcParams {
   int32_t M;             // valid rows of X
+  int32_t rows_per_seq;  // the block holds M / rows_per_seq sequences, sequence-major
   int32_t N;             // output features (for masking the last tile)
   int32_t K;
   int32_t n_pad;         // MMA N: rows of X padded to a multiple of 16
@@ -119,7 +120,9 @@ struct GemmTcParams {
   bf16* kc;              // this layer's key cache   [H_kv][C_max][D]
   bf16* vc;              // this layer's value cache
   const float2* rope_blk;  // (cos, sin) [row][D/2] for the block's position ids
-  const int32_t* len_ptr;  // cache length C (device)
+  const int32_t* len_ptr;  // cache length C of the block's first sequence (device); the next sequence's `len_stride` ints on
+  int32_t len_stride;
+  long long seq_stride;    // elements between the cache slabs of consecutive sequences (kc, vc point at the first one's)
   int32_t H, H_kv, D, C_max;
 };
 
@@ -300,7 +303,6 @@ __device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const floa
                                                int cnt, int warp, int lane, AllIn all_in) {
   constexpr int NW = TC_THREADS / 32;
   const int n4 = tile * TC_BLOCK_N + 4 * lane;               // first output feature of the quad
-  const int C = p.mode == EPI_QKV ? *p.len_ptr : 0;
   float g4[4] = {1.f, 1.f, 1.f, 1.f};
   if (p.mode == EPI_RESID && n4 + 3 < p.N) {
     const uint2 gv = *reinterpret_cast<const uint2*>(p.gain + n4);
@@ -413,7 +415,7 @@ __device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const floa
         for (int u = 0; u < RB; ++u) {
           if (!live[u]) continue;                              // warp-uniform
           const int row = t0 + tb + NW * u;
-          const int kk = p.row_kind[row] == ROW_MASK ? p.k_max : 1;
+          const int kk = p.row_kind[row % p.rows_per_seq] == ROW_MASK ? p.k_max : 1;
           unsigned long long key[4];
           const float vals[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
 #pragma unroll
@@ -493,13 +495,18 @@ __device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const floa
           pk.y = pack_bf16x2(r.z, r.w);
           if (!live[u]) continue;
           const int tok = t0 + tb + NW * u;
-          const int slot = C + tok;
           if (head < p.H) {
             *reinterpret_cast<uint2*>(p.q + ((size_t)tok * p.H + head) * p.D + dd) = pk;
-          } else if (slot < p.C_max) {
-            bf16* base = head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
-                                             : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D;
-            *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
+          } else {
+            // row `rs` of sequence `sq` goes to slot C(sq) + rs of that sequence's cache slab
+            const int sq = tok / p.rows_per_seq, rs = tok - sq * p.rows_per_seq;
+            const int slot = p.len_ptr[(size_t)sq * p.len_stride] + rs;
+            if (slot < p.C_max) {
+              bf16* base = (head < p.H + p.H_kv ? p.kc + (size_t)(head - p.H) * p.C_max * p.D
+                                                : p.vc + (size_t)(head - p.H - p.H_kv) * p.C_max * p.D) +
+                           (size_t)sq * p.seq_stride;
+              *reinterpret_cast<uint2*>(base + (size_t)slot * p.D + dd) = pk;
+            }
           }
         }
       }

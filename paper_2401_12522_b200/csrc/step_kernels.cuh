@@ -15,8 +15,9 @@ namespace bita {
 // Packing (Sec. 3.2, Appendix B: the candidate tree and its mask groups become one row sequence):
 // row 0 = last accepted token, rows 1..N = tree tokens (token -1 -> zero row), then the mask
 // embeddings.  Position ids: C + rel_pos.
-// x: fp32 [M][d] residual stream; pos: int32 [M].
-__global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int32_t* __restrict__ tree_tokens,
+// x: fp32 [B * M][d] residual stream; pos: int32 [B * M].  `states`: the context's per-sequence
+// states; `tree_tokens`: [B][N] or null (each sequence's own drafted tree).
+__global__ void k_embed(DevPlan plan, const DevState* __restrict__ states, const int32_t* __restrict__ tree_tokens,
                         const int32_t* __restrict__ query_tokens, const bf16* __restrict__ tok_emb,
                         const bf16* __restrict__ mask_emb, int d, int V, float* __restrict__ x,
                         int32_t* __restrict__ pos, int32_t* __restrict__ row_token,
@@ -25,18 +26,20 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
                         unsigned long long* __restrict__ sumsq, int n_slots) {
   pdl_launch();
   pdl_wait();
-  const int r = blockIdx.x;
-  const int kind = plan.row_kind[r];
-  const int idx = plan.row_idx[r];
+  const int r = blockIdx.x;                              // global row
+  const int b = r / plan.M, rs = r - b * plan.M;         // sequence of the block, row within it
+  const DevState* st = states + plan.seq0 + b;
+  const int kind = plan.row_kind[rs];
+  const int idx = plan.row_idx[rs];
   const bf16* src = nullptr;
   int tok = -1;
   if (kind == ROW_ROOT) tok = st->root;
-  else if (kind == ROW_NODE) tok = tree_tokens ? tree_tokens[idx] : st->tree[idx];
+  else if (kind == ROW_NODE) tok = tree_tokens ? tree_tokens[(size_t)b * plan.N + idx] : st->tree[idx];
   else if (kind == ROW_QUERY) tok = query_tokens[idx];
   if (kind == ROW_MASK) src = mask_emb + (size_t)idx * d;
   else if (tok >= 0 && tok < V) src = tok_emb + (size_t)tok * d;
   if (threadIdx.x == 0) {
-    pos[r] = st->len + plan.rel_pos[r];
+    pos[r] = st->len + plan.rel_pos[rs];
     row_token[r] = (tok >= 0 && tok < V) ? tok : -1;
   }
   float* xr = x + (size_t)r * d;
@@ -61,7 +64,7 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
   }
   for (int sl = 1 + threadIdx.x; sl < n_slots; sl += blockDim.x) sumsq[(size_t)sl * BITA_MAX_ROWS + r] = 0ull;
   // (cos, sin) row of this row's position id, for the rotary embedding in the q/k/v projection
-  const int p = st->len + plan.rel_pos[r];
+  const int p = st->len + plan.rel_pos[rs];
   for (int j = threadIdx.x; j < half; j += blockDim.x) rope_blk[(size_t)r * half + j] = rope_tab[(size_t)p * half + j];
 }
 
@@ -70,15 +73,15 @@ __global__ void k_embed(DevPlan plan, const DevState* __restrict__ st, const int
 // of a token row, the top k predictions of a mask row): every tile of 128 vocabulary entries has
 // left its best entries of each row as ordered keys; one block per row picks the overall best
 // k of them, again one at a time ("the largest key below the previous pick").
-// cand: [M][tiles][BITA_MAX_TOPK]; sel_id / sel_val as k_select writes them.
+// cand: [rows][tiles][BITA_MAX_TOPK]; sel_id, sel_val: [rows][BITA_MAX_TOPK], best first.
 __global__ void __launch_bounds__(256) k_select_merge(DevPlan plan, const unsigned long long* __restrict__ cand, int tiles,
                                                       int32_t* __restrict__ sel_id, float* __restrict__ sel_val) {
   pdl_launch();
   pdl_wait();
   __shared__ unsigned long long red[8];
   __shared__ unsigned long long pick;
-  const int r = blockIdx.x;
-  const int K = plan.row_kind[r] == ROW_MASK ? plan.k_max : 1;
+  const int r = blockIdx.x;                              // global row
+  const int K = plan.row_kind[r % plan.M] == ROW_MASK ? plan.k_max : 1;
   const unsigned long long* row = cand + (size_t)r * tiles * BITA_MAX_TOPK;
   const int n = tiles * K;                           // entry e: tile e / K, slot e % K
   unsigned long long prev = ~0ull;
@@ -109,13 +112,20 @@ __global__ void __launch_bounds__(256) k_select_merge(DevPlan plan, const unsign
 // ---------------------------------------------------------------------------------------------
 // Greedy verification (Algorithm 1, else-branch, general-tree form) and next-tree construction
 // (Algorithm 1, last step of the else-branch: the next candidates are the top-k picks of the mask
-// group that hangs on the last accepted node).  One warp: lanes scan the children of the current node.
-__global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t* __restrict__ row_token,
-                         const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec) {
+// group that hangs on the last accepted node).  One warp per sequence of the block (grid = B): lanes
+// scan the children of the current node.  Sequences accept independently: each has its own tree
+// tokens, walk, accepted length and next tree.
+__global__ void k_accept(DevPlan plan, DevState* __restrict__ states, const int32_t* __restrict__ row_token_all,
+                         const int32_t* __restrict__ sel_id_all, DevRecord* __restrict__ recs) {
   pdl_launch();
   pdl_wait();
   const int lane = threadIdx.x;
   const int N = plan.N;
+  const int b = blockIdx.x;
+  DevState* st = states + plan.seq0 + b;
+  DevRecord* rec = recs + plan.seq0 + b;
+  const int32_t* row_token = row_token_all + (size_t)b * plan.M;
+  const int32_t* sel_id = sel_id_all + (size_t)b * plan.M * BITA_MAX_TOPK;
   int cur = -1;
   int a = sel_id[0];
   int n_acc = 0;
@@ -162,7 +172,7 @@ __global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t*
     rec->n_acc = n_acc;
     rec->old_len = C;
     rec->new_len = C + 1 + n_acc;
-    rec->status = st->status;
+    rec->status = states[0].status;                     // the context's one sticky status word
     st->len = C + 1 + n_acc;
     st->root = a;
   }
@@ -170,11 +180,13 @@ __global__ void k_accept(DevPlan plan, DevState* __restrict__ st, const int32_t*
 
 // First pass (Algorithm 1, t = 1): the last query row's argmax is emitted, the one mask group that
 // follows it drafts the first tree.  `last` = this is the final chunk of the query.
-__global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __restrict__ st,
-                                 const int32_t* __restrict__ sel_id, DevRecord* __restrict__ rec, int last) {
+__global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __restrict__ states,
+                                 const int32_t* __restrict__ sel_id, DevRecord* __restrict__ recs, int last) {
   pdl_launch();
   pdl_wait();
   const int lane = threadIdx.x;
+  DevState* st = states + chunk.seq0;                    // the first pass takes one sequence at a time
+  DevRecord* rec = recs + chunk.seq0;
   const int C = st->len;
   const int T = chunk.n_query;
   __syncwarp();
@@ -197,7 +209,7 @@ __global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __r
       rec->n_acc = 0;
       rec->old_len = C;
       rec->new_len = C + T;
-      rec->status = st->status;
+      rec->status = states[0].status;
       st->root = a;
     }
   }
@@ -208,16 +220,19 @@ __global__ void k_prefill_finish(DevPlan chunk, DevPlan step_plan, DevState* __r
 // Cache compaction (Fig. 3 caption: rejected drafts and what follows them leave no trace): the
 // j-th accepted node's entry moves from slot C+1+idx_j to slot C+1+j.  One thread
 // owns a 16-byte column chunk and walks j upwards, which is alias-safe because idx_j >= j and
-// idx is increasing along a path.  grid = (L * H_kv), cache layout [L][H_kv][C_max][D].
-__global__ void k_compact(const DevRecord* __restrict__ rec, int D, int C_max, bf16* __restrict__ kc,
+// idx is increasing along a path.  grid = (L * H_kv, B), cache layout [L][B][H_kv][C_max][D]: every
+// sequence moves its own accepted entries (a different number per sequence) inside its own slabs.
+__global__ void k_compact(const DevRecord* __restrict__ recs, int D, int C_max, int H_kv, int B, bf16* __restrict__ kc,
                           bf16* __restrict__ vc) {
   pdl_launch();
   pdl_wait();
+  const DevRecord* rec = recs + blockIdx.y;
   const int n_acc = rec->n_acc;
   if (n_acc == 0) return;
   const int C = rec->old_len;
   const int chunks = D / 8;                       // 16-byte chunks per row
-  const size_t base = (size_t)blockIdx.x * C_max * D;
+  const int l = blockIdx.x / H_kv, h = blockIdx.x - l * H_kv;
+  const size_t base = (((size_t)l * B + blockIdx.y) * H_kv + h) * C_max * D;
   for (int t = threadIdx.x; t < 2 * chunks; t += blockDim.x) {
     bf16* buf = (t < chunks ? kc : vc) + base;
     const int c = (t < chunks ? t : t - chunks) * 8;
@@ -244,16 +259,17 @@ __global__ void k_wait_probe(int32_t* __restrict__ status, unsigned long long li
   if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, status, limit_ns);
 }
 
-__global__ void k_set_state(DevState* st, int len, int root) {
+__global__ void k_set_state(DevState* st, int len, int root) {   // st: the state of ONE sequence
   pdl_launch();
   pdl_wait();
   if (threadIdx.x == 0) { st->len = len; st->root = root; }
   for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
 }
 
-__global__ void k_reset_state(DevState* st) {
+__global__ void k_reset_state(DevState* states) {                 // grid = sequences of the context
   pdl_launch();
   pdl_wait();
+  DevState* st = states + blockIdx.x;
   if (threadIdx.x == 0) { st->len = 0; st->root = -1; st->status = 0; st->pad = 0; }
   for (int x = threadIdx.x; x < BITA_MAX_NODES; x += blockDim.x) st->tree[x] = -1;
 }

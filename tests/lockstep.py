@@ -47,7 +47,9 @@ def rel_l2(a: np.ndarray, b: np.ndarray) -> float:
 
 class Lockstep:
     def __init__(self, shape, seed: int, template, *, C_max: int, device="cuda:0", lazy_oracle=False,
-                 check_hidden=True, tol: Tolerances = TARGET, weights=None, model=None):
+                 check_hidden=True, tol: Tolerances = TARGET, weights=None, model=None, gpu=None, seq: int = 0):
+        """`gpu`, `seq`: compare sequence `seq` of an existing context of several sequences (the
+        caller drives that context's passes and hands each sequence's record to `after_step`)."""
         from paper_2401_12522_b200 import Bita
 
         self.shape, self.template, self.tol = shape, template, tol
@@ -60,9 +62,13 @@ class Lockstep:
             self.model = oracle_model(shape, seed)
         self.blk = block_for(template, shape.n_mask)
         self.st = orc.State(self.model)
-        self.gpu = Bita(shape, w, template, C_max=C_max, device=device)
+        self.seq = seq
+        self.row0 = 0             # first row of this sequence in the debug buffers of the pass being compared
+        self.owns_gpu = gpu is None
+        self.gpu = Bita(shape, w, template, C_max=C_max, device=device) if gpu is None else gpu
         self.check_hidden = check_hidden
-        self.gpu.enable_debug(True)
+        if self.owns_gpu:
+            self.gpu.enable_debug(True)
         self.adopted = 0          # passes where a sub-tolerance choice of the GPU was adopted
         self.exact = 0            # passes where every margin was above tolerance and records matched bit for bit
         self.layer_err = np.zeros(shape.L)    # per layer, worst pass: error the layer adds (see Tolerances)
@@ -89,14 +95,18 @@ class Lockstep:
 
     # ------------------------------------------------------------------ pieces
     def _gpu_hidden(self, l: int, rows: int) -> np.ndarray:
-        return self.gpu.debug_hidden(l, rows).cpu().numpy().astype(np.float64)
+        return self.gpu.debug_hidden(l, self.row0 + rows)[self.row0:].cpu().numpy().astype(np.float64)
+
+    def _slab(self, cache: torch.Tensor, l: int) -> torch.Tensor:
+        """[H_kv][C_max][D] of this sequence in layer l (the cache of a batch context has a sequence axis)."""
+        return cache[l] if cache.dim() == 4 else cache[l, self.seq]
 
     def _layer_on_gpu_input(self, l, lw, rows, x0, pos, C, vis, sees_prompt) -> np.ndarray:
         """The oracle's layer l applied to the GPU's own input of that layer (its residual stream
         after layer l - 1, its cache as context)."""
         x_in = x0 if l == 0 else self._gpu_hidden(l - 1, rows)
-        ck = self.gpu.k_cache[l, :, :C, :].double().cpu().numpy()
-        cv = self.gpu.v_cache[l, :, :C, :].double().cpu().numpy()
+        ck = self._slab(self.gpu.k_cache, l)[:, :C, :].double().cpu().numpy()
+        cv = self._slab(self.gpu.v_cache, l)[:, :C, :].double().cpu().numpy()
         return orc._layer(self.model, lw, x_in, pos, ck, cv, vis, sees_prompt)[0]
 
     def _observe_layers(self, rows, x0, pos, C, vis, sees_prompt) -> Optional[Dict]:
@@ -135,7 +145,7 @@ class Lockstep:
                 self.acc_err[l] = max(self.acc_err[l], acc)
                 assert own <= tol.layer_rel_l2, f"hidden layer {l}: the layer adds rel L2 {own:.3e} (allowed {tol.layer_rel_l2:.1e})"
                 assert acc <= tol.hidden_rel_l2, f"hidden layer {l}: accumulated rel L2 {acc:.3e} (allowed {tol.hidden_rel_l2:.1e})"
-        gl = self.gpu.debug_logits(rows).cpu().numpy()
+        gl = self.gpu.debug_logits(self.row0 + rows)[self.row0:].cpu().numpy()
         ol = rec_o["logits"]
         rms = float(np.sqrt(np.mean(ol * ol)))
         err = float(np.abs(gl.astype(np.float64) - ol).max()) / rms
@@ -167,14 +177,15 @@ class Lockstep:
         L = self.shape.L
         for l in range(L):
             for name, gcache, ocache in (("k", self.gpu.k_cache, self.st.k), ("v", self.gpu.v_cache, self.st.v)):
-                g = gcache[l, :, since:upto, :].float().cpu().numpy().astype(np.float64)
+                g = self._slab(gcache, l)[:, since:upto, :].float().cpu().numpy().astype(np.float64)
                 o = ocache[l][:, since:upto, :]
                 e = rel_l2(g, o)
                 assert e <= self.tol.kv_rel_l2, f"cache {name} layer {l}: rel L2 {e:.3e}"
 
     # ------------------------------------------------------------------ passes
     def prefill(self, prompt: Sequence[int]):
-        rec_g = self.gpu.prefill(prompt)
+        rec_g = self.gpu.prefill(prompt, seq=self.seq)
+        self.row0 = 0             # the first pass takes one sequence at a time: its rows start the buffers
         T = len(prompt)
         n = self.shape.n_mask
         # the library runs the first pass in equal blocks of at most MAX_ROWS - 8 query rows; the debug
@@ -229,6 +240,13 @@ class Lockstep:
         toks = list(self.st.tree if tree_tokens is None else tree_tokens)
         C0 = self.st.C
         rec_g = self.gpu.step(None if tree_tokens is None else toks)
+        return self.after_step(rec_g, toks, C0)
+
+    def after_step(self, rec_g: Dict, toks: Sequence[int], C0: int, row0: int = 0):
+        """Compares one sequence's share of a finished pass (its record, its rows of the debug
+        buffers from `row0` on, its cache) with the oracle's pass from the same state."""
+        blk = self.blk
+        self.row0 = row0
         layer_in = (blk.M, orc.embed_block(self.model, blk, self.st.root, toks), C0 + blk.rel_pos, C0, blk.vis,
                     blk.sees_prompt)
         teacher = self._observe_layers(*layer_in)
@@ -272,6 +290,38 @@ class Lockstep:
         self._check_cache(self.st.C, since=C0)
         self.emitted.extend(out)
         return rec_g
+
+    def close(self):
+        if self.owns_gpu:
+            self.gpu.close()
+
+
+class BatchLockstep:
+    """Several sequences decoded together by one context, each compared with its own oracle run:
+    every sequence has its own prompt (different lengths), cache, tree and accepted length."""
+
+    def __init__(self, shape, seed: int, template, batch: int, *, C_max: int, device="cuda:0", tol: Tolerances = TARGET,
+                 lazy_oracle=False, weights=None):
+        from paper_2401_12522_b200 import Bita
+        w = weights if weights is not None else synth.make_weights(shape, seed, dtype=torch.bfloat16, device=device)
+        self.gpu = Bita(shape, w, template, C_max=C_max, device=device, batch=batch)
+        self.gpu.enable_debug(True)
+        model = oracle_model_from_device(shape, w) if lazy_oracle else oracle_model(shape, seed)
+        self.seqs = [Lockstep(shape, seed, template, C_max=C_max, device=device, tol=tol, weights=w, model=model,
+                              gpu=self.gpu, seq=b) for b in range(batch)]
+        self.M = self.seqs[0].blk.M
+
+    def prefill(self, prompts: Sequence[Sequence[int]]):
+        return [ls.prefill(p) for ls, p in zip(self.seqs, prompts)]
+
+    def step(self, trees: Optional[Sequence[Optional[Sequence[int]]]] = None):
+        """`trees`: per sequence a token list, or None = all sequences verify the trees they drafted."""
+        toks = [list(ls.st.tree) for ls in self.seqs] if trees is None else [list(t) for t in trees]
+        C0 = [ls.st.C for ls in self.seqs]
+        recs = self.gpu.step_batch(None if trees is None else toks)
+        for b, ls in enumerate(self.seqs):
+            ls.after_step(recs[b], toks[b], C0[b], row0=b * self.M)
+        return recs
 
     def close(self):
         self.gpu.close()

@@ -34,7 +34,7 @@ def test_struct_sizes_match_header_constants():
     text = open(os.path.join(ROOT, "include", "bita.h")).read()
     consts = {k: int(v) for k, v in re.findall(r"#define (BITA_MAX_[A-Z]+) (\d+)", text)}
     assert consts == {"BITA_MAX_NODES": b.MAX_NODES, "BITA_MAX_ROWS": b.MAX_ROWS, "BITA_MAX_DEPTH": b.MAX_DEPTH,
-                      "BITA_MAX_TOPK": b.MAX_TOPK, "BITA_MAX_MASK": b.MAX_MASK}
+                      "BITA_MAX_TOPK": b.MAX_TOPK, "BITA_MAX_MASK": b.MAX_MASK, "BITA_MAX_BATCH": b.MAX_BATCH}
     assert C.sizeof(b.StepOut) == 4 * (3 + b.MAX_DEPTH + 1 + b.MAX_DEPTH + b.MAX_NODES)
     assert C.sizeof(b.ModelDims) == 44
 
@@ -79,6 +79,12 @@ def test_host_side_validation():
     # rank beyond the top-k width
     tm5, keep5 = _tmpl([-1], [16], [-1])
     assert lib.bita_workspace_bytes(C.byref(d), C.byref(tm5), shape.n_mask, C.byref(need)) == -2
+    # several sequences: the rows of all of them share one block (19 rows each here)
+    assert lib.bita_workspace_bytes_batch(C.byref(d), C.byref(tm), shape.n_mask, 16, C.byref(need)) == 0
+    assert lib.bita_workspace_bytes_batch(C.byref(d), C.byref(tm), shape.n_mask, 17, C.byref(need)) == -1
+    assert lib.bita_workspace_bytes_batch(C.byref(d), C.byref(tm), shape.n_mask, 0, C.byref(need)) == -1
+    assert lib.bita_workspace_bytes_batch(C.byref(d), C.byref(tm4), 4, 2, C.byref(need)) == -2     # 2 x 325 rows
+    assert lib.bita_step_batch(None, None, None, C.byref(out0 := b.StepOut())) == -1
     # null context
     out = b.StepOut()
     assert lib.bita_step(None, None, None, C.byref(out)) == -1
