@@ -358,12 +358,16 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
   return BITA_OK;
 }
 
-// Split-K factor a launch of `g` takes for a block of n_pad padded rows: blocks past 128 padded
-// rows run one CTA per SM, and then a split only pays while all its CTAs fit in one wave.
+// Blocks of up to this many padded rows run two CTAs per SM (two accumulators of up to 256 columns
+// share the SM's tensor memory, two rings its shared memory); larger ones one CTA per SM.
+constexpr int TWO_PER_SM_MAX_ROWS = 256;
+
+// Split-K factor a launch of `g` takes for a block of n_pad padded rows: with one CTA per SM a
+// split only pays while all its CTAs fit in one wave.
 int effective_splits(const GemmDesc& g, int n_pad) {
   const int sms = sm_count();
   int splits = g.splits;
-  if (n_pad > 128 && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
+  if (n_pad > TWO_PER_SM_MAX_ROWS && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
   return splits;
 }
 
@@ -372,7 +376,8 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
                    cudaStream_t stream) {
   DeviceFacts* facts = device_facts();
   if (!facts->gemm_attr) {
-    CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
     facts->gemm_attr = true;
   }
   if (!p.wait_ns) p.wait_ns = TC_WAIT_LIMIT_NS;
@@ -383,21 +388,27 @@ int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M
   while (cols < n_pad) cols <<= 1;
   p.tmem_cols = cols;
   const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  // Blocks of up to 128 padded rows run two CTAs per SM (half the shared memory each: 4 ring stages
-  // up to 96 rows, 3 beyond); larger ones one per SM, and then a split only pays while all its CTAs
-  // fit in one wave.
+  // Two CTAs per SM take half the shared memory each: 4 ring stages up to 96 rows, 3 up to 160,
+  // 2 beyond.
   const int sms = sm_count();
-  const bool two_per_sm = n_pad <= 128 && g.tiles * splits > sms;
+  const bool two_per_sm = n_pad <= TWO_PER_SM_MAX_ROWS && g.tiles * splits > sms;
   const size_t budget = (two_per_sm ? 110 : 220) * 1024;
   const size_t extra = 1024;                                 // alignment slack
   int stages = (int)((budget - extra) / stage);
   if (stages > 10) stages = 10;
   if (stages < 2) stages = 2;
-  if ((size_t)stages * stage < (size_t)M * TC_BLOCK_N * 4) return BITA_ERR_INVALID_ARG;   // staging of a whole tile
+  // an unsplit tile is finished from a staging copy in the ring's memory: all rows at once if they fit, else 96 at a time
+  {
+    const int fit = (int)((size_t)stages * stage / ((size_t)TC_BLOCK_N * 4));
+    p.stg_rows = fit >= M ? M : fit / 96 * 96;
+    if (p.stg_rows < 1) return BITA_ERR_INVALID_ARG;
+  }
   p.splits = splits;
   p.stages = stages;
   const size_t smem = stages * stage + extra;
-  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc, g.a0, g.a1, map_b, p);
+  if (splits == 1 && p.stg_rows < M)
+    return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc<true>, g.a0, g.a1, map_b, p);
+  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc<false>, g.a0, g.a1, map_b, p);
 }
 
 // Padded row count of a block as the MMA sees it: a multiple of 16; past 256 rows a multiple of 32,

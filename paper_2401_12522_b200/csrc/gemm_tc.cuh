@@ -87,6 +87,7 @@ struct GemmTcParams {
   int32_t K;
   int32_t n_pad;         // MMA N: rows of X padded to a multiple of 16
   int32_t stages;
+  int32_t stg_rows;      // splits == 1: rows of the tile staged in shared memory at a time (a multiple of 96, or M)
   int32_t splits;        // split-K factor = gridDim.y
   int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1
   int32_t tmem_cols;     // power of two >= max(32, n_pad)
@@ -514,6 +515,9 @@ __device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const floa
   }
 }
 
+// CHUNKED: an unsplit tile whose rows do not fit the ring's memory all at once is finished
+// p.stg_rows rows at a time (read back, fused operation, next rows); otherwise in one go.
+template <bool CHUNKED>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
           const __grid_constant__ CUtensorMap map_b, GemmTcParams p) {
@@ -644,7 +648,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
 
   // ---------------- epilogue, part 1: accumulator -> staging
   // splits == 1: the tile goes to shared memory (`stg`, the pipeline stages, free once the
-  //              accumulator barrier has completed), row-major [M][128] fp32.
+  //              accumulator barrier has completed), row-major [rows][128] fp32 (all M rows, or
+  //              p.stg_rows at a time in the CHUNKED instance).
   // splits  > 1: every split stores its partial tile to the global exchange buffer
   //              part[tile][split][M][128] (L2-resident, overwritten by every projection) and
   //              counts itself in; once all splits of the tile are in, each of them sums an equal
@@ -668,7 +673,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     float* dst = p.splits > 1 ? part_tile + (size_t)split * tile_elems : stg;
     ok = __all_sync(0xffffffffu, ok);                          // the TMEM loads below are warp-wide
     const uint32_t lane_addr = tmem_base + ((uint32_t)(lg * 32) << 16);
-    for (int c = 0; c < p.n_pad; c += 96) {                    // up to 96 columns per TMEM round trip
+    const int c_end = CHUNKED ? min(p.n_pad, p.stg_rows) : p.n_pad;   // CHUNKED: the first rows only
+    for (int c = 0; c < c_end; c += 96) {                      // up to 96 columns per TMEM round trip
       float v[96];
       const int groups = min(3, (p.n_pad - c + 31) >> 5);      // 32-column groups, inside the allocation
       if (nkb > 0 && ok) {
@@ -690,10 +696,39 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   // Rows of the tile this CTA finishes: all of them without a split, else an equal share, so that
   // the reduction and the fused operation of a tile are spread over all its splits.
   const int t0 = p.splits > 1 ? (int)((long)p.M * split / p.splits) : 0;
-  const int cnt = (p.splits > 1 ? (int)((long)p.M * (split + 1) / p.splits) : p.M) - t0;
+  const int cnt = (p.splits > 1 ? (int)((long)p.M * (split + 1) / p.splits) : (CHUNKED ? min(p.M, p.stg_rows) : p.M)) - t0;
   pdl_wait();
   if (p.splits == 1) {
     fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, [] {});
+    if constexpr (CHUNKED) {
+      // the remaining rows, p.stg_rows (a multiple of 96) at a time through the same staging memory
+      for (int c0 = p.stg_rows; c0 < p.M; c0 += p.stg_rows) {
+        const int c1 = min(c0 + p.stg_rows, p.M);
+        __syncthreads();                                       // the staging rows are rewritten
+        if (warp >= 2) {
+          const int fr = (warp & 3) * 32 + lane;
+          const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+          for (int c = c0; c < c1; c += 96) {
+            float v[96];
+            const int groups = min(3, (p.n_pad - c + 31) >> 5);
+            if (nkb > 0) {
+              if (groups == 1) tmem_ld32(lane_addr + (uint32_t)c, v);
+              else if (groups == 2) tmem_ld64(lane_addr + (uint32_t)c, v);
+              else tmem_ld96(lane_addr + (uint32_t)c, v);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 96; ++j) v[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 96; ++j)
+              if (j < groups * 32 && c + j < p.M) stg[(c + j - c0) * TC_BLOCK_N + fr] = v[j];
+          }
+        }
+        tc_fence_before();
+        __syncthreads();
+        fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, c0, c1 - c0, warp, lane, [] {});
+      }
+    }
   } else {
     int32_t* arrived = p.tile_counters + tile;
     if (threadIdx.x == 0) {
