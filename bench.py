@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) per projection launch at the 7B width with the 69-row block, from the ncu
 # capture summarised in profiles/k_gemm_tc_k_attn_umma_7b_ncu_full.md (q/k/v, O, gate/up, down per
 # layer; LM head).  Other shapes have no capture: their `traffic` is null.
-NCU_TRAFFIC_7B = {"per_layer": 105.57e6 + 35.54e6 + 184.55e6 + 96.89e6, "head": 266.14e6}
+NCU_TRAFFIC_7B = {"per_layer": 105.16e6 + 35.45e6 + 184.81e6 + 96.93e6, "head": 266.94e6}
 
 
 def _traffic_per_mean_launch(shape, tmpl):
