@@ -278,6 +278,8 @@ int make_map3(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64
 // One weight matrix (or a gate/up pair) as the projection kernel sees it.
 struct GemmDesc {
   CUtensorMap a0, a1;
+  CUtensorMap a0w, a1w;   // the same matrices with boxes of 128 rows (wide tiles); for a single matrix a0w = a0
+  int max_splits = 8;
   const void *w0 = nullptr, *w1 = nullptr;
   int N = 0, K = 0, dual = 0, tiles = 0, splits = 1;
   int kind = 0;           // which set of split-arrival counters its launches count on (GemmKind)
@@ -347,73 +349,146 @@ int make_gemm_desc(GemmDesc* g, const void* W0, const void* W1, int N, int K, in
     g->N = N;
     if ((rc = make_map(&g->a0, W0, K, N, 64))) return rc;
     if ((rc = make_map(&g->a1, W1, K, N, 64))) return rc;
+    if ((rc = make_map(&g->a0w, W0, K, N, TC_BLOCK_N))) return rc;
+    if ((rc = make_map(&g->a1w, W1, K, N, TC_BLOCK_N))) return rc;
   } else {
     g->tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
     g->N = N;
     if ((rc = make_map(&g->a0, W0, K, N, TC_BLOCK_N))) return rc;
     g->a1 = g->a0;
+    g->a0w = g->a0;
+    g->a1w = g->a0;
   }
+  g->max_splits = max_splits;
   if (g->tiles > TC_MAX_TILES) return BITA_ERR_INVALID_ARG;
   g->splits = gemm_splits(g->tiles, K, max_splits);
   return BITA_OK;
 }
 
+// Padded row count of a block as the MMA sees it: a multiple of 16; past 256 rows a multiple of 32,
+// so that each of the two column halves is a multiple of 16.
+inline int pad16(int m) { return m <= 16 ? 16 : (m <= 256 ? (m + 15) / 16 * 16 : (m + 31) / 32 * 32); }
+
 // Blocks of up to this many padded rows run two CTAs per SM (two accumulators of up to 256 columns
 // share the SM's tensor memory, two rings its shared memory); larger ones one CTA per SM.
 constexpr int TWO_PER_SM_MAX_ROWS = 256;
 
-// Split-K factor a launch of `g` takes for a block of n_pad padded rows: with one CTA per SM a
-// split only pays while all its CTAs fit in one wave.
-int effective_splits(const GemmDesc& g, int n_pad) {
-  const int sms = sm_count();
-  int splits = g.splits;
-  if (n_pad > TWO_PER_SM_MAX_ROWS && g.tiles * splits > sms) splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
-  return splits;
+// How a projection is launched for a block of n_pad padded rows (M valid ones).
+struct GemmPlan {
+  bool wide = false;      // 256 weight rows per CTA (two accumulators), see k_gemm_tc
+  bool chunked = false;   // unsplit tile finished stg_rows rows at a time
+  int tiles = 0;          // gridDim.x
+  int splits = 1;         // gridDim.y
+  int stages = 2;
+  int stg_rows = 0;
+  int tmem_cols = 32;
+  size_t smem = 0;
+};
+
+// 0 = never, 1 = wherever the shapes allow, -1 (default) = where it pays: launches whose narrow
+// tiles would need a second wave of CTAs.
+int wide_policy() {
+  static const int v = [] {
+    const char* e = getenv("BITA_WIDE_TILES");
+    return e ? atoi(e) : -1;
+  }();
+  return v;
 }
+
+GemmPlan plan_gemm(const GemmDesc& g, int n_pad, int M) {
+  GemmPlan pl;
+  const int sms = sm_count();
+  const int kb = (g.K + TC_BLOCK_K - 1) / TC_BLOCK_K;
+  const size_t extra = 1024;                                   // alignment slack
+  // ---- narrow: 128 weight rows per CTA
+  auto narrow = [&]() {
+    GemmPlan n;
+    n.tiles = g.tiles;
+    n.splits = g.splits;
+    // with one CTA per SM a split only pays while all its CTAs fit in one wave
+    if (n_pad > TWO_PER_SM_MAX_ROWS && g.tiles * n.splits > sms) n.splits = sms / g.tiles > 0 ? sms / g.tiles : 1;
+    int cols = 32;
+    while (cols < n_pad) cols <<= 1;
+    n.tmem_cols = cols;
+    const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
+    // Two CTAs per SM take half the shared memory each: 4 ring stages up to 96 rows, 3 up to 160, 2 beyond.
+    const bool two_per_sm = n_pad <= TWO_PER_SM_MAX_ROWS && g.tiles * n.splits > sms;
+    const size_t budget = (two_per_sm ? 110 : 220) * 1024;
+    int stages = (int)((budget - extra) / stage);
+    if (stages > 10) stages = 10;
+    if (stages < 2) stages = 2;
+    n.stages = stages;
+    // an unsplit tile is finished from a staging copy in the ring's memory: all rows at once if they fit, else 96 at a time
+    const int fit = (int)((size_t)stages * stage / ((size_t)TC_BLOCK_N * 4));
+    n.stg_rows = fit >= M ? M : fit / 96 * 96;
+    n.chunked = n.splits == 1 && n.stg_rows < M;
+    n.smem = stages * stage + extra;
+    return n;
+  };
+  pl = narrow();
+  const int policy = wide_policy();
+  if (policy == 0 || n_pad > 256 || g.tiles < 2) return pl;
+  // ---- wide: 256 weight rows per CTA, half the CTAs
+  GemmPlan w;
+  w.wide = true;
+  w.tiles = (g.tiles + 1) / 2;
+  const bool small = n_pad <= 128;                             // two accumulators of <= 128 columns: two CTAs per SM possible
+  int s = (small ? 2 * sms : sms) / w.tiles;
+  if (s > kb / 4) s = kb / 4;
+  if (s > g.max_splits) s = g.max_splits;
+  if (s > GEMM_MAX_SPLITS) s = GEMM_MAX_SPLITS;
+  if (s < 1) s = 1;
+  w.splits = s;
+  int cols = 32;
+  while (cols < 2 * n_pad) cols <<= 1;
+  w.tmem_cols = cols;
+  const size_t stage = (size_t)2 * TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
+  const bool two_per_sm = small && w.tiles * s > sms;
+  const size_t budget = (two_per_sm ? 110 : 220) * 1024;
+  int stages = (int)((budget - extra) / stage);
+  if (stages > 10) stages = 10;
+  if (stages < 2) return pl;
+  w.stages = stages;
+  w.stg_rows = M;
+  if (s == 1 && (size_t)stages * stage < (size_t)2 * M * TC_BLOCK_N * 4) return pl;   // both accumulators are staged whole
+  if (w.tiles * s > (small ? 2 * sms : sms)) return pl;        // the wide launch itself must be one wave
+  w.smem = stages * stage + extra;
+  if (policy == 1) return w;
+  // default: only where the narrow launch does not fit the GPU at once
+  const int slots = n_pad <= TWO_PER_SM_MAX_ROWS ? 2 * sms : sms;
+  return pl.tiles * pl.splits > slots ? w : pl;
+}
+
+int effective_splits(const GemmDesc& g, int n_pad, int M) { return plan_gemm(g, n_pad, M).splits; }
 
 // Launch: X bf16 (first M rows valid) times the described weights; `p` carries the epilogue.
 int launch_gemm_tc(const GemmDesc& g, const CUtensorMap& map_b, int n_pad, int M, GemmTcParams p, bool pdl,
                    cudaStream_t stream) {
   DeviceFacts* facts = device_facts();
   if (!facts->gemm_attr) {
-    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
-    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
+    CU_TRY(cudaFuncSetAttribute(k_gemm_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
     facts->gemm_attr = true;
   }
   if (!p.wait_ns) p.wait_ns = TC_WAIT_LIMIT_NS;
-  int splits = effective_splits(g, n_pad);
+  const GemmPlan pl = plan_gemm(g, n_pad, M);
   p.M = M; p.N = g.N; p.K = g.K; p.n_pad = n_pad; p.dual = g.dual;
+  p.n_vtiles = g.tiles;
   if (p.rows_per_seq < 1) p.rows_per_seq = M;
-  int cols = 32;
-  while (cols < n_pad) cols <<= 1;
-  p.tmem_cols = cols;
-  const size_t stage = (size_t)TC_BLOCK_N * TC_BLOCK_K * 2 + (size_t)n_pad * TC_BLOCK_K * 2;
-  // Two CTAs per SM take half the shared memory each: 4 ring stages up to 96 rows, 3 up to 160,
-  // 2 beyond.
-  const int sms = sm_count();
-  const bool two_per_sm = n_pad <= TWO_PER_SM_MAX_ROWS && g.tiles * splits > sms;
-  const size_t budget = (two_per_sm ? 110 : 220) * 1024;
-  const size_t extra = 1024;                                 // alignment slack
-  int stages = (int)((budget - extra) / stage);
-  if (stages > 10) stages = 10;
-  if (stages < 2) stages = 2;
-  // an unsplit tile is finished from a staging copy in the ring's memory: all rows at once if they fit, else 96 at a time
-  {
-    const int fit = (int)((size_t)stages * stage / ((size_t)TC_BLOCK_N * 4));
-    p.stg_rows = fit >= M ? M : fit / 96 * 96;
-    if (p.stg_rows < 1) return BITA_ERR_INVALID_ARG;
-  }
-  p.splits = splits;
-  p.stages = stages;
-  const size_t smem = stages * stage + extra;
-  if (splits == 1 && p.stg_rows < M)
-    return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc<true>, g.a0, g.a1, map_b, p);
-  return launch(stream, pdl, dim3(g.tiles, splits), dim3(TC_THREADS), smem, 1, k_gemm_tc<false>, g.a0, g.a1, map_b, p);
+  p.tmem_cols = pl.tmem_cols;
+  p.stg_rows = pl.stg_rows;
+  if (p.stg_rows < 1) return BITA_ERR_INVALID_ARG;
+  p.splits = pl.splits;
+  p.stages = pl.stages;
+  const dim3 grid(pl.tiles, pl.splits);
+  if (pl.wide)
+    return launch(stream, pdl, grid, dim3(TC_THREADS), pl.smem, 1, k_gemm_tc<false, true>, g.a0w, g.a1w, map_b, p);
+  if (pl.chunked)
+    return launch(stream, pdl, grid, dim3(TC_THREADS), pl.smem, 1, k_gemm_tc<true, false>, g.a0, g.a1, map_b, p);
+  return launch(stream, pdl, grid, dim3(TC_THREADS), pl.smem, 1, k_gemm_tc<false, false>, g.a0, g.a1, map_b, p);
 }
 
-// Padded row count of a block as the MMA sees it: a multiple of 16; past 256 rows a multiple of 32,
-// so that each of the two column halves is a multiple of 16.
-inline int pad16(int m) { return m <= 16 ? 16 : (m <= 256 ? (m + 15) / 16 * 16 : (m + 31) / 32 * 32); }
 
 // Attention launch shape: row tiles (one CTA takes one tile of 128 query rows, or two when the block
 // has more than 128 rows), and key slices.  The slices of a (sequence,
@@ -469,8 +544,8 @@ size_t carve(const bita_model_dims& m, uint8_t* base, Buffers* b) {
   const size_t S = 8;                        // upper bound of attn_splits
   t.part_ml = (float*)take((size_t)m.H * S * R * 2 * 4);
   t.part_acc = (float*)take((size_t)m.H * S * R * m.D * 4);
-  t.gemm_part = (float*)take((size_t)GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);
-  t.gemm_cnt = (int32_t*)take((size_t)GEMM_KINDS * TC_MAX_TILES * 4);
+  t.gemm_part = (float*)take((size_t)2 * GEMM_MAX_CTAS * R * TC_BLOCK_N * 4);   // a wide CTA leaves two partial tiles
+  t.gemm_cnt = (int32_t*)take((size_t)2 * GEMM_KINDS * TC_MAX_TILES * 4);
   t.rope_tab = (float2*)take((size_t)(m.C_max + 64) * (m.D / 2) * sizeof(float2));
   t.rope_blk = (float2*)take(R * (size_t)(m.D / 2) * sizeof(float2));
   t.state = (DevState*)take(sizeof(DevState) * BITA_MAX_BATCH);      // one per sequence
@@ -504,7 +579,7 @@ struct bita_ctx {
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;   // (buffer, K, padded rows) -> map
   std::map<std::tuple<const void*, const void*, const void*, const void*, int, int, int, int>, AttnMaps> attn_map_cache;
   bool pdl;                             // programmatic dependent launch between the kernels of a pass
-  uint32_t split_arrivals[GEMM_KINDS];  // what every counter of a set has reached once the launches so far are done
+  uint32_t split_arrivals[2 * GEMM_KINDS];  // what every counter of a set has reached once the launches so far are done
   unsigned long long wait_ns;           // bound of every device-side wait
   int last_rows;                        // rows of the most recent pass (what the debug buffer holds)
 
@@ -551,11 +626,13 @@ int gemm(bita_ctx* c, const GemmDesc& g, const bf16* X, int M, GemmTcParams p) {
   p.status = &c->b.state->status;
   p.wait_ns = c->wait_ns;
   p.part = c->b.gemm_part;
-  p.tile_counters = c->b.gemm_cnt + (size_t)g.kind * TC_MAX_TILES;
   {
-    const int splits = effective_splits(g, n_pad);
-    if (splits > 1) c->split_arrivals[g.kind] += (uint32_t)splits;
-    p.arrive_target = (int32_t)c->split_arrivals[g.kind];
+    // wide and narrow launches of a kind count on sets of their own (they cover different tile ranges)
+    const GemmPlan pl = plan_gemm(g, n_pad, M);
+    const int set = g.kind + (pl.wide ? GEMM_KINDS : 0);
+    p.tile_counters = c->b.gemm_cnt + (size_t)set * TC_MAX_TILES;
+    if (pl.splits > 1) c->split_arrivals[set] += (uint32_t)pl.splits;
+    p.arrive_target = (int32_t)c->split_arrivals[set];
   }
   mark(c, 0);
   int rc = launch_gemm_tc(g, it->second, n_pad, M, p, c->pdl, c->stream);
@@ -865,8 +942,8 @@ int bita_init_batch(bita_ctx** out, const bita_model_dims* dims, const bita_weig
   }
   rc = upload_plan(&c->step_plan, c->b.plan_step, c->stream);
   if (rc) return fail(rc);
-  if (cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
-  for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
+  if (cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)2 * GEMM_KINDS * TC_MAX_TILES * 4, c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
+  for (int k = 0; k < 2 * GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
   k_reset_state<<<BITA_MAX_BATCH, 128, 0, c->stream>>>(c->b.state);
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(BITA_ERR_CUDA);
   *out = c;
@@ -883,8 +960,8 @@ int bita_batch(const bita_ctx* c) { return c ? c->B : BITA_ERR_INVALID_ARG; }
 int bita_reset(bita_ctx* c, bita_kv* kv) {
   if (!c || !kv) return BITA_ERR_INVALID_ARG;
   // a pass that gave up on a wait may have left split counters half way
-  CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)GEMM_KINDS * TC_MAX_TILES * 4, c->stream));
-  for (int k = 0; k < GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
+  CU_TRY(cudaMemsetAsync(c->b.gemm_cnt, 0, (size_t)2 * GEMM_KINDS * TC_MAX_TILES * 4, c->stream));
+  for (int k = 0; k < 2 * GEMM_KINDS; ++k) c->split_arrivals[k] = 0;
   k_reset_state<<<BITA_MAX_BATCH, 128, 0, c->stream>>>(c->b.state);
   CU_TRY(cudaStreamSynchronize(c->stream));
   c->prefilled.assign(c->B, 0);
@@ -1114,9 +1191,13 @@ int bita_last_cuda_error(void) { return g_last_cuda_error; }
 // Workspace of the stand-alone projection: status word, tile counters, split-K exchange buffer.
 int bita_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K, size_t* out_bytes) {
   if (!out_bytes || M < 1 || M > BITA_MAX_ROWS || N < 1 || K < 8 || K % 8) return BITA_ERR_INVALID_ARG;
-  const int tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
-  const int splits = gemm_splits(tiles, K, 8);
-  *out_bytes = ALIGN + align_up((size_t)tiles * 4) + align_up(splits > 1 ? (size_t)tiles * splits * M * TC_BLOCK_N * 4 : 0);
+  GemmDesc g;                                                  // shape only: the plan needs no tensor maps
+  g.N = N; g.K = K; g.max_splits = 8;
+  g.tiles = (N + TC_BLOCK_N - 1) / TC_BLOCK_N;
+  g.splits = gemm_splits(g.tiles, K, 8);
+  const GemmPlan pl = plan_gemm(g, pad16(M), M);
+  const size_t part_tiles = (size_t)pl.tiles * (pl.wide ? 2 : 1) * pl.splits;       // partial tiles of 128 features
+  *out_bytes = ALIGN + align_up((size_t)g.tiles * 4) + align_up(pl.splits > 1 ? part_tiles * M * TC_BLOCK_N * 4 : 0);
   return BITA_OK;
 }
 
@@ -1139,7 +1220,7 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   p.status = (int32_t*)workspace;
   p.tile_counters = (int32_t*)((uint8_t*)workspace + ALIGN);
   p.part = (float*)((uint8_t*)workspace + ALIGN + cnt_bytes);
-  p.arrive_target = effective_splits(g, n_pad);                    // the counters were just cleared
+  p.arrive_target = effective_splits(g, n_pad, M);                 // the counters were just cleared
   if ((rc = launch_gemm_tc(g, mb, n_pad, M, p, false, s))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;

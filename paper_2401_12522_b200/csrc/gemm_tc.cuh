@@ -89,7 +89,8 @@ struct GemmTcParams {
   int32_t stages;
   int32_t stg_rows;      // splits == 1: rows of the tile staged in shared memory at a time (a multiple of 96, or M)
   int32_t splits;        // split-K factor = gridDim.y
-  int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1
+  int32_t dual;          // 1: tile = 64 rows of map A0 + 64 rows of map A1 (wide instance: 128 + 128)
+  int32_t n_vtiles;      // wide instance: 128-feature "virtual" tiles of the whole launch (a CTA finishes two)
   int32_t tmem_cols;     // power of two >= max(32, n_pad)
   int32_t mode;          // GemmEpilogue
   int32_t* status;       // device status word (sticky error flag)
@@ -517,7 +518,13 @@ __device__ __forceinline__ void fused_epilogue(const GemmTcParams& p, const floa
 
 // CHUNKED: an unsplit tile whose rows do not fit the ring's memory all at once is finished
 // p.stg_rows rows at a time (read back, fused operation, next rows); otherwise in one go.
-template <bool CHUNKED>
+// WIDE: a CTA takes 256 weight rows (two boxes of 128: consecutive rows of one matrix, or the
+// matching 128 rows of a gate/up pair) against ONE activation tile: two MMAs per K step into two
+// accumulators of n_pad columns (n_pad <= 256).  Half the CTAs for the same weights, and the
+// activation tile is fetched once per 32 KiB of weights instead of once per 16 KiB.  The
+// accumulators are finished as two "virtual" tiles of 128 features each (virtual tile 2 * tile + j),
+// which is exactly what the narrow instance would have produced for them.
+template <bool CHUNKED, bool WIDE>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
           const __grid_constant__ CUtensorMap map_b, GemmTcParams p) {
@@ -536,7 +543,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   const int nkb = kb1 - kb0;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t a_bytes = TC_BLOCK_N * TC_BLOCK_K * 2;                 // 16 KiB
+  static_assert(!(CHUNKED && WIDE), "the wide instance stages whole tiles");
+  constexpr int NH = WIDE ? 2 : 1;                                      // accumulators (boxes of 128 weight rows) per CTA
+  const uint32_t a_bytes = NH * TC_BLOCK_N * TC_BLOCK_K * 2;            // 16 KiB per box
   const uint32_t b_bytes = (uint32_t)p.n_pad * TC_BLOCK_K * 2;
   const uint32_t stage_bytes = a_bytes + b_bytes;
 
@@ -577,7 +586,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
         const int kx = (kb0 + i) * TC_BLOCK_K;
         mbar_expect_tx(full, stage_bytes);
-        if (p.dual) {
+        if constexpr (WIDE) {
+          const int r0 = p.dual ? tile * TC_BLOCK_N : tile * 2 * TC_BLOCK_N;
+          tma_load_2d(sa, &map_a0, kx, r0, full, pol_w);
+          if (p.dual) tma_load_2d(sa + a_bytes / 2, &map_a1, kx, r0, full, pol_w);
+          else tma_load_2d(sa + a_bytes / 2, &map_a0, kx, r0 + TC_BLOCK_N, full, pol_w);
+        } else if (p.dual) {
           tma_load_2d(sa, &map_a0, kx, row_a, full, pol_w);
           tma_load_2d(sa + a_bytes / 2, &map_a1, kx, row_a, full, pol_w);
         } else {
@@ -638,6 +652,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
             // advancing 16 elements along K = 32 bytes = 2 units of the descriptor's address field
             umma_bf16(tmem_base + (uint32_t)(h * n_half), da + (uint64_t)(2 * k), dbh + (uint64_t)(2 * k), idesc,
                       (i > 0 || k > 0) ? 1u : 0u);
+            if constexpr (WIDE)     // second box of weight rows (16 KiB further), second accumulator (n_pad columns further)
+              umma_bf16(tmem_base + (uint32_t)p.n_pad, da + (uint64_t)((TC_BLOCK_N * TC_BLOCK_K * 2) >> 4) + (uint64_t)(2 * k),
+                        dbh + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
           }
         }
         umma_commit(smem_u32(&bar_empty[s]));                 // frees the stage when these MMAs are done
@@ -657,7 +674,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   //              the fused operation to those rows.
   float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
   const size_t tile_elems = (size_t)p.M * TC_BLOCK_N;
-  float* part_tile = p.part + (size_t)tile * p.splits * tile_elems;      // this tile's partials, split-major
+  float* part_tile = p.part + (size_t)tile * NH * p.splits * tile_elems;  // this tile's partials: [virtual tile][split]
   if (warp >= 2) {
     const int lg = warp & 3;                                   // TMEM lane group this warp may read
     const int fr = lg * 32 + lane;                             // feature row of the tile owned by this thread
@@ -670,24 +687,55 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     bool ok = true;
     if (nkb > 0) ok = mbar_wait(smem_u32(&bar_acc), 0, p.status, p.wait_ns);
     tc_fence_after();
-    float* dst = p.splits > 1 ? part_tile + (size_t)split * tile_elems : stg;
-    ok = __all_sync(0xffffffffu, ok);                          // the TMEM loads below are warp-wide
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(lg * 32) << 16);
-    const int c_end = CHUNKED ? min(p.n_pad, p.stg_rows) : p.n_pad;   // CHUNKED: the first rows only
-    for (int c = 0; c < c_end; c += 96) {                      // up to 96 columns per TMEM round trip
-      float v[96];
-      const int groups = min(3, (p.n_pad - c + 31) >> 5);      // 32-column groups, inside the allocation
-      if (nkb > 0 && ok) {
-        if (groups == 1) tmem_ld32(lane_addr + (uint32_t)c, v);
-        else if (groups == 2) tmem_ld64(lane_addr + (uint32_t)c, v);
-        else tmem_ld96(lane_addr + (uint32_t)c, v);
-      } else {
+    if constexpr (!WIDE) {
+      float* dst = p.splits > 1 ? part_tile + (size_t)split * tile_elems : stg;
+      ok = __all_sync(0xffffffffu, ok);                          // the TMEM loads below are warp-wide
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(lg * 32) << 16);
+      const int c_end = CHUNKED ? min(p.n_pad, p.stg_rows) : p.n_pad;   // CHUNKED: the first rows only
+      for (int c = 0; c < c_end; c += 96) {                      // up to 96 columns per TMEM round trip
+        float v[96];
+        const int groups = min(3, (p.n_pad - c + 31) >> 5);      // 32-column groups, inside the allocation
+        if (nkb > 0 && ok) {
+          if (groups == 1) tmem_ld32(lane_addr + (uint32_t)c, v);
+          else if (groups == 2) tmem_ld64(lane_addr + (uint32_t)c, v);
+          else tmem_ld96(lane_addr + (uint32_t)c, v);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 96; ++j) v[j] = 0.f;
+          for (int j = 0; j < 96; ++j) v[j] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 96; ++j)
+          if (j < groups * 32 && c + j < p.M) dst[(c + j) * TC_BLOCK_N + fr] = v[j];
       }
+    } else {
+      ok = __all_sync(0xffffffffu, ok);                          // the TMEM loads below are warp-wide
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(lg * 32) << 16);
+      const int c_end = CHUNKED ? min(p.n_pad, p.stg_rows) : p.n_pad;   // CHUNKED: the first rows only
 #pragma unroll
-      for (int j = 0; j < 96; ++j)
-        if (j < groups * 32 && c + j < p.M) dst[(c + j) * TC_BLOCK_N + fr] = v[j];
+      for (int hv = 0; hv < NH; ++hv) {
+        // Where feature row `fr` of accumulator hv goes: virtual tile vj, column vc of its 128.  A wide
+        // gate/up pair (accumulator 0 = 128 gate rows, 1 = the matching up rows) is laid out as two
+        // pair tiles of 64 + 64, the layout the SwiGLU operation expects.
+        int vj = hv, vc = fr;
+        if (WIDE && p.dual) { vj = fr >> 6; vc = hv * 64 + (fr & 63); }
+        float* dst = p.splits > 1 ? part_tile + ((size_t)vj * p.splits + split) * tile_elems : stg + (size_t)vj * tile_elems;
+        for (int c = 0; c < c_end; c += 96) {                    // up to 96 columns per TMEM round trip
+          float v[96];
+          const int groups = min(3, (p.n_pad - c + 31) >> 5);    // 32-column groups, inside the allocation
+          if (nkb > 0 && ok) {
+            const uint32_t ta = lane_addr + (uint32_t)(hv * p.n_pad + c);
+            if (groups == 1) tmem_ld32(ta, v);
+            else if (groups == 2) tmem_ld64(ta, v);
+            else tmem_ld96(ta, v);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 96; ++j) v[j] = 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 96; ++j)
+            if (j < groups * 32 && c + j < p.M) dst[(c + j) * TC_BLOCK_N + vc] = v[j];
+        }
+      }
     }
   }
   tc_fence_before();
@@ -698,70 +746,121 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
   const int t0 = p.splits > 1 ? (int)((long)p.M * split / p.splits) : 0;
   const int cnt = (p.splits > 1 ? (int)((long)p.M * (split + 1) / p.splits) : (CHUNKED ? min(p.M, p.stg_rows) : p.M)) - t0;
   pdl_wait();
-  if (p.splits == 1) {
-    fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, [] {});
-    if constexpr (CHUNKED) {
-      // the remaining rows, p.stg_rows (a multiple of 96) at a time through the same staging memory
-      for (int c0 = p.stg_rows; c0 < p.M; c0 += p.stg_rows) {
-        const int c1 = min(c0 + p.stg_rows, p.M);
-        __syncthreads();                                       // the staging rows are rewritten
-        if (warp >= 2) {
-          const int fr = (warp & 3) * 32 + lane;
-          const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-          for (int c = c0; c < c1; c += 96) {
-            float v[96];
-            const int groups = min(3, (p.n_pad - c + 31) >> 5);
-            if (nkb > 0) {
-              if (groups == 1) tmem_ld32(lane_addr + (uint32_t)c, v);
-              else if (groups == 2) tmem_ld64(lane_addr + (uint32_t)c, v);
-              else tmem_ld96(lane_addr + (uint32_t)c, v);
-            } else {
+  if constexpr (!WIDE) {
+    if (p.splits == 1) {
+      fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, t0, cnt, warp, lane, [] {});
+      if constexpr (CHUNKED) {
+        // the remaining rows, p.stg_rows (a multiple of 96) at a time through the same staging memory
+        for (int c0 = p.stg_rows; c0 < p.M; c0 += p.stg_rows) {
+          const int c1 = min(c0 + p.stg_rows, p.M);
+          __syncthreads();                                       // the staging rows are rewritten
+          if (warp >= 2) {
+            const int fr = (warp & 3) * 32 + lane;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            for (int c = c0; c < c1; c += 96) {
+              float v[96];
+              const int groups = min(3, (p.n_pad - c + 31) >> 5);
+              if (nkb > 0) {
+                if (groups == 1) tmem_ld32(lane_addr + (uint32_t)c, v);
+                else if (groups == 2) tmem_ld64(lane_addr + (uint32_t)c, v);
+                else tmem_ld96(lane_addr + (uint32_t)c, v);
+              } else {
 #pragma unroll
-              for (int j = 0; j < 96; ++j) v[j] = 0.f;
+                for (int j = 0; j < 96; ++j) v[j] = 0.f;
+              }
+#pragma unroll
+              for (int j = 0; j < 96; ++j)
+                if (j < groups * 32 && c + j < p.M) stg[(c + j - c0) * TC_BLOCK_N + fr] = v[j];
             }
-#pragma unroll
-            for (int j = 0; j < 96; ++j)
-              if (j < groups * 32 && c + j < p.M) stg[(c + j - c0) * TC_BLOCK_N + fr] = v[j];
           }
+          tc_fence_before();
+          __syncthreads();
+          fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, c0, c1 - c0, warp, lane, [] {});
         }
-        tc_fence_before();
-        __syncthreads();
-        fused_epilogue<6, 0>(p, stg, nullptr, tile_elems, rstd_s, tile, (int)gridDim.x, c0, c1 - c0, warp, lane, [] {});
       }
+    } else {
+      int32_t* arrived = p.tile_counters + tile;
+      if (threadIdx.x == 0) {
+        __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
+        atomicAdd(arrived, 1);
+      }
+      // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
+      // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+      // The counter is never reset: the host tells each launch the value that means "all in", so no
+      // split has to report that it has finished reading (the exchange buffer is next written by a
+      // later kernel, which starts its own stores only after this one has completed).
+      auto all_in = [&]() {
+        if (threadIdx.x == 0) {
+          unsigned long long w0 = 0;
+          bool ok = true;
+          for (uint32_t spin = 0; (int32_t)((uint32_t)ld_acquire_gpu(arrived) - (uint32_t)p.arrive_target) < 0; ++spin) {
+            if ((spin & 63u) == 63u) {
+              const unsigned long long now = global_ns();
+              if (w0 == 0) w0 = now;
+              else if (now - w0 > p.wait_ns) { ok = false; break; }
+            }
+          }
+          if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
+          __threadfence();
+        }
+        __syncthreads();
+      };
+      // rows per batch x loads per row in flight, sized so that a 69..128-row block takes one batch
+      const int nt = (int)gridDim.x;
+      if (p.splits == 2) fused_epilogue<6, 2>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+      else if (p.splits == 3) fused_epilogue<4, 3>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+      else if (p.splits == 4) fused_epilogue<4, 4>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+      else fused_epilogue<2, 8>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
     }
   } else {
-    int32_t* arrived = p.tile_counters + tile;
-    if (threadIdx.x == 0) {
-      __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
-      atomicAdd(arrived, 1);
-    }
-    // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
-    // before it has published its own partial tile: the wait ends, and it is bounded all the same.
-    // The counter is never reset: the host tells each launch the value that means "all in", so no
-    // split has to report that it has finished reading (the exchange buffer is next written by a
-    // later kernel, which starts its own stores only after this one has completed).
-    auto all_in = [&]() {
-      if (threadIdx.x == 0) {
-        unsigned long long w0 = 0;
-        bool ok = true;
-        for (uint32_t spin = 0; (int32_t)((uint32_t)ld_acquire_gpu(arrived) - (uint32_t)p.arrive_target) < 0; ++spin) {
-          if ((spin & 63u) == 63u) {
-            const unsigned long long now = global_ns();
-            if (w0 == 0) w0 = now;
-            else if (now - w0 > p.wait_ns) { ok = false; break; }
-          }
-        }
-        if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
-        __threadfence();
+    const int nt = p.n_vtiles;                                  // 128-feature tiles of the launch
+    if (p.splits == 1) {
+#pragma unroll
+      for (int vj = 0; vj < NH; ++vj) {
+        const int vt = tile * NH + vj;
+        if (vt < nt) fused_epilogue<6, 0>(p, stg + (size_t)vj * tile_elems, nullptr, tile_elems, rstd_s, vt, nt, t0, cnt, warp, lane, [] {});
       }
-      __syncthreads();
-    };
-    // rows per batch x loads per row in flight, sized so that a 69..128-row block takes one batch
-    const int nt = (int)gridDim.x;
-    if (p.splits == 2) fused_epilogue<6, 2>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
-    else if (p.splits == 3) fused_epilogue<4, 3>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
-    else if (p.splits == 4) fused_epilogue<4, 4>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
-    else fused_epilogue<2, 8>(p, nullptr, part_tile, tile_elems, rstd_s, tile, nt, t0, cnt, warp, lane, all_in);
+    } else {
+      int32_t* arrived = p.tile_counters + tile;
+      if (threadIdx.x == 0) {
+        __threadfence();                                         // the CTA's partial tile (ordered by the barrier above) before the count
+        atomicAdd(arrived, 1);
+      }
+      // The splits of a tile are CTAs of one wave (the host sizes the grid so), none of which waits
+      // before it has published its own partial tile: the wait ends, and it is bounded all the same.
+      // The counter is never reset: the host tells each launch the value that means "all in", so no
+      // split has to report that it has finished reading (the exchange buffer is next written by a
+      // later kernel, which starts its own stores only after this one has completed).
+      auto all_in = [&]() {
+        if (threadIdx.x == 0) {
+          unsigned long long w0 = 0;
+          bool ok = true;
+          for (uint32_t spin = 0; (int32_t)((uint32_t)ld_acquire_gpu(arrived) - (uint32_t)p.arrive_target) < 0; ++spin) {
+            if ((spin & 63u) == 63u) {
+              const unsigned long long now = global_ns();
+              if (w0 == 0) w0 = now;
+              else if (now - w0 > p.wait_ns) { ok = false; break; }
+            }
+          }
+          if (!ok) atomicExch(p.status, BITA_ERR_TIMEOUT);
+          __threadfence();
+        }
+        __syncthreads();
+      };
+      // rows per batch x loads per row in flight, sized so that a 69..128-row block takes one batch
+      bool waited = false;
+#pragma unroll
+      for (int vj = 0; vj < NH; ++vj) {
+        const int vt = tile * NH + vj;
+        const float* pt = part_tile + (size_t)vj * p.splits * tile_elems;
+        auto once = [&]() { if (!waited) { all_in(); waited = true; } };   // the tile's splits are waited for once
+        if (vt >= nt) { once(); continue; }
+        if (p.splits == 2) fused_epilogue<6, 2>(p, nullptr, pt, tile_elems, rstd_s, vt, nt, t0, cnt, warp, lane, once);
+        else if (p.splits == 3) fused_epilogue<4, 3>(p, nullptr, pt, tile_elems, rstd_s, vt, nt, t0, cnt, warp, lane, once);
+        else if (p.splits == 4) fused_epilogue<4, 4>(p, nullptr, pt, tile_elems, rstd_s, vt, nt, t0, cnt, warp, lane, once);
+        else fused_epilogue<2, 8>(p, nullptr, pt, tile_elems, rstd_s, vt, nt, t0, cnt, warp, lane, once);
+      }
+    }
   }
   __syncthreads();
   if (warp == 1) {

@@ -24,7 +24,9 @@ def test_generators_are_bit_identical_on_cpu_and_gpu():
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (19, 1376, 256), (19, 256, 688), (69, 1000, 4096),
                                    (133, 384, 1024), (256, 130, 520), (105, 4096, 4096), (128, 4096, 2048),
                                    (154, 4096, 4096), (200, 1000, 11008), (256, 12288, 4096),
-                                   (260, 1000, 512), (325, 4096, 4096), (340, 300, 11008), (352, 12288, 4096)])
+                                   (260, 1000, 512), (325, 4096, 4096), (340, 300, 11008), (352, 12288, 4096),
+                                   # more 128-row tiles than CTA slots: 256 weight rows per CTA (even / odd tile count)
+                                   (69, 40960, 512), (69, 38016, 256), (128, 38016, 512)])
 def test_projection_matches_fp64_matmul(M, N, K):
     from paper_2401_12522_b200 import bita_gemm_bf16
     X = synth.pseudo_normal(3, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda:0")
