@@ -34,16 +34,22 @@ METRIC = "accepted_tokens_per_s"
 UNIT = "tokens/s"
 
 
-# DRAM bytes (read + write) per projection launch at the 7B width with the 69-row block, from the ncu
-# capture summarised in profiles/k_gemm_tc_k_attn_umma_7b_ncu_full.md (q/k/v, O, gate/up, down per
-# layer; LM head).  Other shapes have no capture: their `traffic` is null.
-NCU_TRAFFIC_7B = {"per_layer": 105.16e6 + 35.45e6 + 184.81e6 + 96.93e6, "head": 266.94e6}
+# DRAM bytes (read + write) per projection launch with the 69-row block (q/k/v, O, gate/up, down per
+# layer; LM head), from the ncu captures of small cases of the same kernels summarised in
+# profiles/k_gemm_tc_k_attn_umma_7b_ncu_full.md and profiles/k_gemm_tc_70b_width_ncu_full.md (one or two
+# layers of the width; traffic per launch does not depend on the depth, so a pass is L x the layer's
+# launches + the head's).  The 13B width has no capture: its `traffic` is null.
+NCU_TRAFFIC = {
+    "7b": {"per_layer": 105.16e6 + 35.45e6 + 184.81e6 + 96.93e6, "head": 266.94e6},
+    "70b": {"per_layer": 173.88e6 + 141.25e6 + 944.74e6 + 480.06e6, "head": 529.02e6},
+}
 
 
 def _traffic_per_mean_launch(shape, tmpl):
-    if not shape.name.startswith("7b") or (1 + tmpl.N + tmpl.G * shape.n_mask) != 69:
+    t = NCU_TRAFFIC.get(shape.name.split("-")[0])
+    if t is None or (1 + tmpl.N + tmpl.G * shape.n_mask) != 69:
         return None
-    return (shape.L * NCU_TRAFFIC_7B["per_layer"] + NCU_TRAFFIC_7B["head"]) / (4 * shape.L + 1)
+    return (shape.L * t["per_layer"] + t["head"]) / (4 * shape.L + 1)
 
 
 def _peaks():
