@@ -261,6 +261,14 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
  * for it, and a second kernel merges.)  A wait between key slices that runs out (2 s) leaves
  * wrong output rather than a hang. */
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes);
+/* The same for a cache of capacity C_max, never less than the above.  With a long cache (16384 keys and
+ * more) and a workspace of this size, bita_tree_attention may cut the keys into as many slices (up to
+ * 64) as make the waves of CTAs come out even - e.g. 8 sequences x 32 heads are 256 CTAs, two uneven
+ * waves on 148 SMs, but 1024 CTAs of a quarter of the keys each are seven even ones - and merges the
+ * slices' partial results with its second kernel.  With the smaller workspace the call still works,
+ * with the cluster shape. */
+int bita_attention_workspace_bytes_long(int32_t B, int32_t M, int32_t H, int32_t D, int32_t C_max,
+                                        size_t* out_bytes);
 /* Diagnostic, process-wide: 0 (default) = key slices merge inside a thread-block cluster whenever
  * that launch form is accepted; 1 = always through the workspace and the separate merge kernel.
  * Affects bita_tree_attention and the passes of every context. */

@@ -81,6 +81,7 @@ def _signatures():
         "bita_gemm_workspace_bytes": [i32, i32, i32, C.POINTER(sz)],
         "bita_gemm_bf16": [vp, vp, vp, i32, i32, i32, vp, sz, vp],
         "bita_attention_workspace_bytes": [i32, i32, i32, i32, C.POINTER(sz)],
+        "bita_attention_workspace_bytes_long": [i32, i32, i32, i32, i32, C.POINTER(sz)],
         "bita_tree_attention": [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp],
         "bita_tree_attention_static": [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp],
     }
@@ -318,15 +319,17 @@ def bita_tree_attention(q, k, v, vis, prompt_k, prompt_v, sees_prompt, ctx_len, 
     B, M, H, D = q.shape
     C_max = k.shape[2]
     need = C.c_size_t(0)
-    _check(lib.bita_attention_workspace_bytes(B, M, H, D, C.byref(need)), "bita_attention_workspace_bytes")
+    _check(lib.bita_attention_workspace_bytes_long(B, M, H, D, C_max, C.byref(need)),
+           "bita_attention_workspace_bytes_long")
     if workspace is None and need.value:
         workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=q.device)
     wp = 0 if workspace is None else (workspace.data_ptr() + 255) // 256 * 256
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size() - (wp - workspace.data_ptr())
     if out is None:
         out = torch.empty((B, M, H * D), dtype=torch.bfloat16, device=q.device)
     _check(lib.bita_tree_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(vis), _ptr(prompt_k), _ptr(prompt_v),
                                    _ptr(sees_prompt), _ptr(ctx_len), _ptr(out), B, M, H, H_kv, D, P, C_max,
-                                   C.c_void_p(wp), need.value, _stream_handle(stream)), "bita_tree_attention")
+                                   C.c_void_p(wp), max(0, ws_bytes), _stream_handle(stream)), "bita_tree_attention")
     return out
 
 

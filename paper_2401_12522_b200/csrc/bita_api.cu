@@ -512,6 +512,34 @@ int attn_splits(int H, int B, int M) {
   return s;
 }
 
+// Long caches: key slices for the workspace route (partial results in global memory, merged by a
+// second kernel), where the slice count is free: the CTAs of such a launch run in waves of one per
+// SM, and the count is chosen so that the waves come out even.  Cost of a choice in units of "one
+// CTA works through one chunk of 128 keys": waves(groups * S) * ceil(chunks / S), plus the traffic of
+// the partial results (M rows of D + 2 floats per group and slice, written and read once) at the rate
+// the GPU streams keys and values (one chunk = 64 KiB per SM).  Returns 0 when the cluster shape is
+// within 5 % of the best (short caches always: launch latency matters more there).
+constexpr int ATTN_MAX_WS_SLICES = 64;
+int attn_balanced_slices(int H, int B, int M, int D, int C_max) {
+  int rt, s0;
+  attn_shape(H, B, M, &rt, &s0);
+  const int sms = sm_count();
+  const long groups = (long)H * B * rt;
+  const long chunks = (C_max + AU_KEYS - 1) / AU_KEYS + 1;
+  if (chunks < 128) return 0;
+  auto waves = [&](long ctas) { return (ctas + sms - 1) / sms; };
+  const double part_unit = (double)M * (D + 2) * 4 * 2 / ((double)sms * 2 * AU_KEYS * D * 2);   // per group and slice
+  const double base = (double)waves(groups * s0) * ((chunks + s0 - 1) / s0);
+  double best = base;
+  int best_s = 0;
+  for (int s = 1; s <= ATTN_MAX_WS_SLICES; ++s) {
+    if (chunks / s < 4) break;
+    const double cost = (double)waves(groups * s) * ((chunks + s - 1) / s) + (s > 1 ? part_unit * groups * s : 0.0) + 2.0;
+    if (cost < best * 0.95 && (best_s == 0 || cost < best)) { best = cost; best_s = s; }
+  }
+  return best_s;
+}
+
 // Device buffers of a context, carved from the caller's workspace.
 struct Buffers {
   float* x; bf16* xn; bf16* q; bf16* att; bf16* hf; unsigned long long* cand; unsigned long long* sumsq;
@@ -680,9 +708,13 @@ enum { ATTN_ROUTE_AUTO = 0, ATTN_ROUTE_WORKSPACE = 1 };
 int g_attention_route = ATTN_ROUTE_AUTO;      // process-wide diagnostic switch (bita_set_attention_route)
 
 int launch_attention(AttnArgs a, bool pdl, cudaStream_t s, int* n_launched, std::map<AttnMapKey, AttnMaps>* cache,
-                     int route = -1) {
+                     int route = -1, int ws_slices = 0) {
   if (route < 0) route = g_attention_route;
   attn_shape(a.H, a.B, a.M, &a.row_tiles, &a.S);
+  if (ws_slices > 0) {                   // the caller's workspace holds that many slices: even waves, merge kernel
+    a.S = ws_slices;
+    if (ws_slices > 1) route = ATTN_ROUTE_WORKSPACE;
+  }
   AttnMaps maps;
   {
     int rc = attn_maps(a, cache, &maps);
@@ -1226,6 +1258,25 @@ int bita_gemm_bf16(const void* X, const void* W, void* Y, int32_t M, int32_t N, 
   return BITA_OK;
 }
 
+namespace {
+size_t attn_partial_bytes(size_t B, size_t H, size_t S, size_t M, size_t D, size_t* acc_offset) {
+  const size_t ml = align_up(B * H * S * M * 2 * 4);
+  if (acc_offset) *acc_offset = ml;
+  return S <= 1 ? 0 : ml + align_up(B * H * S * M * D * 4);
+}
+}  // namespace
+
+int bita_attention_workspace_bytes_long(int32_t B, int32_t M, int32_t H, int32_t D, int32_t C_max, size_t* out_bytes) {
+  size_t base = 0;
+  int rc = bita_attention_workspace_bytes(B, M, H, D, &base);
+  if (rc) return rc;
+  if (C_max < M) return BITA_ERR_INVALID_ARG;
+  const int s = attn_balanced_slices(H, B, M, D, C_max);
+  const size_t wide = s > 1 ? attn_partial_bytes(B, H, s, M, D, nullptr) : 0;
+  *out_bytes = wide > base ? wide : base;
+  return BITA_OK;
+}
+
 int bita_attention_workspace_bytes(int32_t B, int32_t M, int32_t H, int32_t D, size_t* out_bytes) {
   if (!out_bytes || B < 1 || M < 1 || M > BITA_MAX_ROWS || H < 1 || (D != 64 && D != 128)) return BITA_ERR_INVALID_ARG;
   const size_t S = attn_splits(H, B, M);
@@ -1251,11 +1302,21 @@ int tree_attention_impl(const void* q, const void* k, const void* v, const uint3
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.v = (const bf16*)v; a.vis = vis;
   a.prompt_k = (const bf16*)prompt_k; a.prompt_v = (const bf16*)prompt_v; a.sees_prompt = sees_prompt;
   a.ctx_len = ctx_len; a.ctx_len_stride = 1; a.vis_batch_stride = M * W; a.sp_batch_stride = M; a.out = (bf16*)out;
-  // workspace: partial results of the key slices (used when the slices do not merge inside a cluster)
+  // workspace: partial results of the key slices (used when the slices do not merge inside a cluster).
+  // A long cache with a workspace of bita_attention_workspace_bytes_long takes the slice count that
+  // makes the waves of CTAs come out even.
+  int ws_slices = 0;
+  if (route < 0 && g_attention_route == ATTN_ROUTE_AUTO && workspace && !((uintptr_t)workspace % ALIGN)) {
+    const int s = attn_balanced_slices(H, B, M, D, C_max);
+    if (s > 0 && workspace_bytes >= attn_partial_bytes(B, H, s, M, D, nullptr)) ws_slices = s;
+  }
+  const size_t S_used = ws_slices > 0 ? (size_t)ws_slices : (size_t)attn_splits(H, B, M);
+  size_t acc_off = 0;
+  attn_partial_bytes(B, H, S_used, M, D, &acc_off);
   a.part_ml = (float*)workspace;
-  a.part_acc = (float*)((uint8_t*)a.part_ml + align_up((size_t)B * H * attn_splits(H, B, M) * M * 2 * 4));
+  a.part_acc = (float*)((uint8_t*)a.part_ml + acc_off);
   a.B = B; a.M = M; a.W = W; a.H = H; a.H_kv = H_kv; a.D = D; a.P = P; a.C_max = C_max;
-  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr, route))) return rc;
+  if ((rc = launch_attention(a, false, (cudaStream_t)cuda_stream, nullptr, nullptr, route, ws_slices))) return rc;
   CU_TRY(cudaGetLastError());
   return BITA_OK;
 }

@@ -463,15 +463,22 @@ def test_full_depth_lockstep(name, prompt_len, steps):
     ls.close()
 
 
-@pytest.mark.parametrize("B,N,C", [(1, 128, 32768), (2, 64, 8192), (8, 16, 2048)])
+@pytest.mark.parametrize("B,N,C", [(1, 128, 32768), (2, 64, 8192), (8, 16, 2048), (4, 16, 20000)])
 def test_tree_attention_sweep_shapes(B, N, C):
     """The attention sweep's shapes (32 heads of 128, M = 1 + 4 + N rows); a sample of the outputs
-    is checked against the oracle's attention row by row."""
-    from paper_2401_12522_b200 import bita_tree_attention
+    is checked against the oracle's attention row by row.  The last case (128 CTAs' worth of heads,
+    a long cache) takes the slice count that evens out the waves of CTAs, through the workspace route."""
+    import ctypes as C_
+    from paper_2401_12522_b200 import bita_tree_attention, lib
     H = H_kv = 32
     D, P = 128, 16
     tmpl = synth.random_recursive_template(N + 1, N)
     M = 1 + N + 4
+    if (B, C) == (4, 20000):
+        small, large = C_.c_size_t(0), C_.c_size_t(0)
+        assert lib.bita_attention_workspace_bytes(B, M, H, D, C_.byref(small)) == 0
+        assert lib.bita_attention_workspace_bytes_long(B, M, H, D, C + M + 3, C_.byref(large)) == 0
+        assert small.value == 0 and large.value > 0            # one slice per head by default, several here
     q, k, v, pk, pv, vis, sp, ctx, blk = _random_attention_case(9, B, M, H, H_kv, D, P, C, tmpl)
     out = bita_tree_attention(q, k, v, vis, pk, pv, sp, ctx, H_kv=H_kv, P=P)
     rows = sorted(set([0, 1, M // 2, M - 5, M - 1]))
