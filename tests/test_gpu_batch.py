@@ -8,7 +8,7 @@ import torch
 import synth
 from helpers import block_for, orc, prompt_tokens
 from lockstep import TARGET, BatchLockstep
-from test_gpu_parity import FULL_WIDTH_TOL
+from test_gpu_parity import FULL_WIDTH_TOL, _write_report
 
 pytestmark = pytest.mark.gpu
 
@@ -54,6 +54,7 @@ def test_batch_lockstep_tiny_ragged():
     assert [ls.st.C for ls in bl.seqs] == [len(p) + sum(t[b] for t in lens) for b, p in enumerate(prompts)]
     for ls in bl.seqs:
         assert ls.max_logit <= TARGET.logit_rms and ls.max_hidden_acc <= TARGET.hidden_rel_l2
+        _write_report(ls)
     bl.close()
 
 
@@ -146,4 +147,6 @@ def test_batch_full_width_lockstep(name, batch, prompt_lens):
     trees[1] = synth.plant_tree(tmpl, trees[1], cont, seed, 1, 1.1, shape.V)
     recs = bl.step(trees)
     assert recs[1]["n_out"] >= 2
+    for ls in bl.seqs:
+        _write_report(ls)
     bl.close()
