@@ -150,3 +150,21 @@ def test_batch_full_width_lockstep(name, batch, prompt_lens):
     for ls in bl.seqs:
         _write_report(ls)
     bl.close()
+
+
+def test_rewind_of_one_sequence_leaves_the_others_alone():
+    """bita_rewind_seq cuts one sequence back to an earlier state: that sequence then repeats the pass it
+    took from there (same drafts, same record), the other one carries on from where it was."""
+    from paper_2401_12522_b200 import Bita
+    shape = synth.CONFIGS["tiny"]
+    w = synth.make_weights(shape, 9, dtype=torch.bfloat16, device="cuda:0")
+    tmpl = synth.product_rule_template(shape.tree_K, shape.tree_B)
+    b = Bita(shape, w, tmpl, C_max=256, batch=2)
+    first = [b.prefill(prompt_tokens(9 + s, n, shape.V), seq=s) for s, n in enumerate((30, 41))]
+    r1 = b.step_batch([first[0]["next_tree"], first[1]["next_tree"]])
+    # sequence 1 back to the state after its first pass; sequence 0 stays where the pass left it
+    b.rewind(first[1]["new_len"], first[1]["out_tokens"][-1], seq=1)
+    r2 = b.step_batch([r1[0]["next_tree"], first[1]["next_tree"]])
+    assert r2[1] == r1[1]                                      # the same pass again, bit for bit
+    assert r2[0]["new_len"] == r1[0]["new_len"] + r2[0]["n_out"]
+    b.close()
